@@ -1,0 +1,192 @@
+/*
+ * spsyrk.h - C ABI of the B200 local sparse SYRK library (libspsyrk.so).
+ *
+ * Computes the lower triangle, diagonal included, of the Gram matrix of a sparse matrix,
+ *     C_L = tril(A * A^T),   A in CSR,
+ * without forming the upper half, plus the optional materialisation of the full symmetric
+ * matrix from the computed half and a Jaccard normalisation of intersection counts.
+ *
+ * Conventions
+ *   - Every pointer named d_* is a DEVICE pointer, owned by the caller; h_* and plain
+ *     out-parameters (int64_t *nnz_out, size_t *workspace_bytes, ...) are HOST pointers.
+ *   - The library allocates no device memory except inside spsyrk_host_tril.  Scratch space
+ *     is a caller-owned device workspace whose size is queried first.
+ *   - CSR everywhere: int64 row pointers, int32 column ids, values of the given dtype.  Input
+ *     must be canonical: column ids strictly ascending inside each row (no duplicates) and
+ *     in [0, n).  Output rows are sorted ascending by column id.
+ *   - Stored entries are structural: (i, j) is stored iff rows i and j of A share at least one
+ *     stored column, whatever the value of the sum.  A row of A without entries gives an
+ *     empty output row (no diagonal entry).
+ *   - All device work is enqueued on the CUDA stream passed as `cuda_stream` (a cudaStream_t
+ *     cast to void*; NULL is the default stream).  Functions that hand a value back to the
+ *     host (sizes, nnz, error words) synchronise that stream; the others are asynchronous.
+ *   - Every function returns a status and never throws or aborts.  On error, outputs are
+ *     unspecified.  Limits: m, n < 2^31, nnz(A) < 2^31; nnz of the result is 64-bit.
+ */
+#ifndef SPSYRK_H
+#define SPSYRK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct spsyrk_plan_s *spsyrk_plan_t; /* opaque, created by spsyrk_plan, freed by spsyrk_destroy */
+
+typedef enum {
+    SPSYRK_OK = 0,
+    SPSYRK_ERR_INVALID_ARG = 1,     /* null pointer, negative size, bad enum, bad row range */
+    SPSYRK_ERR_BAD_CSR = 2,         /* row pointers not monotone, column ids unsorted / duplicate / out of range */
+    SPSYRK_ERR_WORKSPACE = 3,       /* workspace smaller than the queried size */
+    SPSYRK_ERR_OVERFLOW = 4,        /* a size exceeds the limits above */
+    SPSYRK_ERR_SEQUENCE = 5,        /* numeric before symbolic, or a stale plan */
+    SPSYRK_ERR_CUDA = 6,            /* a CUDA runtime call failed */
+    SPSYRK_ERR_INTERNAL = 7,        /* a bounded device loop gave up (should not happen) */
+    SPSYRK_ERR_NOT_IMPLEMENTED = 8
+} spsyrk_status_t;
+
+typedef enum { SPSYRK_F64 = 0, SPSYRK_F32 = 1, SPSYRK_I32 = 2 } spsyrk_dtype_t;
+
+/* SPSYRK_TRIL keeps products a_ik * a_jk with j <= i only (Section III-A: a diagonal process
+ * computes only the lower triangle; Algorithm 2, line 2).  SPSYRK_FULL removes the cut-off and
+ * yields all of A * A^T with the same kernels; it exists to measure the work the symmetry saves
+ * (sigma_mul = 1/2 in the cost table of Section III-C). */
+typedef enum { SPSYRK_TRIL = 0, SPSYRK_FULL = 1 } spsyrk_mode_t;
+
+/*
+ * spsyrk_plan - analyse A for output rows [row_begin, row_end).
+ *
+ * Steps (all on the device): validate the CSR; transpose A into column lists whose entries
+ * are ascending by row (the input transpose of Sections III and IV-B, done locally), so that
+ * "rows j <= i of column k" is a prefix of the list; per-row work estimate
+ *     w[i] = sum over nonzeros a_ik of #{entries of column k with row <= i}
+ * (in FULL mode the whole column), whose total is the multiply-add count of Section III-C
+ * (sum_k d_k (d_k + 1) / 2 for the half, sum_k d_k^2 for the full product); binning of the
+ * rows by w into warp / block / large classes.
+ *
+ * Two-phase: call with d_workspace == NULL to receive *workspace_bytes (no device work, *plan
+ * untouched); then call with a buffer of at least that size, 256-byte aligned.  A, the
+ * workspace and the stream's device must outlive the plan; A is read, never written.
+ * The second call synchronises the stream once (validation result and bin sizes).
+ *
+ * Row tiles: plans for disjoint row ranges are independent; concatenating their results gives
+ * the untiled C_L.  (Halving a CSR matrix along rows is free, Section IV-A.)
+ *
+ * d_rowptr[m+1], d_colidx[nnz], d_vals[nnz] of `dtype`.  0 <= row_begin <= row_end <= m.
+ * Errors: INVALID_ARG, OVERFLOW, WORKSPACE, BAD_CSR, CUDA.
+ */
+spsyrk_status_t spsyrk_plan(spsyrk_plan_t *plan, int64_t m, int64_t n, int64_t nnz,
+                            const int64_t *d_rowptr, const int32_t *d_colidx, const void *d_vals,
+                            spsyrk_dtype_t dtype, spsyrk_mode_t mode,
+                            int64_t row_begin, int64_t row_end,
+                            void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
+
+/*
+ * spsyrk_plan_set_rows - re-target an existing plan to another row range of the same A without
+ * repeating the transpose (only the work estimate and the binning are redone).  Invalidates
+ * any symbolic result.  Synchronises the stream once.
+ */
+spsyrk_status_t spsyrk_plan_set_rows(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end,
+                                     void *cuda_stream);
+
+/*
+ * spsyrk_symbolic - count the stored entries of every output row of the plan's range and
+ * turn the counts into row pointers.
+ *   cnt[i] = #{ j <= i : rows i and j of A share a column }   (TRIL; all j in FULL mode)
+ * d_c_rowptr[rows + 1] (rows = row_end - row_begin) receives the exclusive 64-bit prefix sums,
+ * starting at 0 (tile-local).  *nnz_out = d_c_rowptr[rows] is valid on return (one stream
+ * synchronisation).  The lower triangle includes the diagonal (Section V-F).
+ * Errors: INVALID_ARG, INTERNAL, CUDA.
+ */
+spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t *d_c_rowptr, int64_t *nnz_out,
+                                void *cuda_stream);
+
+/*
+ * spsyrk_numeric - fill the rows counted by spsyrk_symbolic.
+ * For each nonzero a_ik of row i and each entry (j, a_jk) of column k with j <= i:
+ * acc[j] += a_ik * a_jk (row-by-row accumulation; Section II-A defines c_ij as the dot product
+ * of rows i and j; Algorithm 2 line 2 restricts it to the lower triangle).  Writes
+ * d_c_colidx[nnz] (global column ids, ascending inside a row) and d_c_vals[nnz] of the plan's
+ * dtype (F32 input is accumulated in double and rounded once; I32 wraps modulo 2^32).
+ * d_c_rowptr must be the array spsyrk_symbolic wrote for this plan.  Asynchronous.
+ * Errors: INVALID_ARG, SEQUENCE, CUDA.
+ */
+spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t *d_c_rowptr,
+                               int32_t *d_c_colidx, void *d_c_vals, void *cuda_stream);
+
+/*
+ * spsyrk_mirror - materialise F = C_L + C_L^T - D, the full symmetric matrix, from a complete
+ * (untiled or re-assembled) lower triangle (Section III-A: "materializes it by transposing";
+ * Section V-F: C = C_L + C_L^T - D).  Row i of F is row i of C_L followed by (r, c_ri) for
+ * every later row r that stores column i, ascending in r; values are bit copies, so F is
+ * exactly symmetric and tril(F) == C_L.
+ *
+ * Three-step use:
+ *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for (m, nnz_l, dtype).
+ *   2. d_f_colidx == NULL: writes d_f_rowptr[m + 1] and *nnz_full_out (synchronises).
+ *   3. all pointers set: fills d_f_colidx / d_f_vals using the d_f_rowptr of step 2.  Asynchronous.
+ * nnz_l = d_l_rowptr[m].  Errors: INVALID_ARG, WORKSPACE, BAD_CSR (an entry above the diagonal), CUDA.
+ */
+spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
+                              const int64_t *d_l_rowptr, const int32_t *d_l_colidx, const void *d_l_vals,
+                              int64_t *d_f_rowptr, int32_t *d_f_colidx, void *d_f_vals,
+                              int64_t *nnz_full_out,
+                              void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
+
+/*
+ * spsyrk_jaccard - Jaccard similarity of the rows of a binary A from intersection counts,
+ *     J_ij = c_ij / (|a_i| + |a_j| - c_ij),   |a_i| = stored entries of row i of A,
+ * for rows [row_begin, row_begin + rows) of an int32-valued C_L with a tile-local row pointer
+ * (Jaccard similarity is the application named in the abstract and Section I; the formula is
+ * the standard set definition).  One single-precision division per stored entry.  Asynchronous.
+ * Errors: INVALID_ARG, CUDA.
+ */
+spsyrk_status_t spsyrk_jaccard(int64_t m, int64_t row_begin, int64_t rows,
+                               const int64_t *d_a_rowptr, const int64_t *d_c_rowptr,
+                               const int32_t *d_c_colidx, const int32_t *d_c_counts,
+                               float *d_jaccard, void *cuda_stream);
+
+/*
+ * spsyrk_plan_stats - host-side facts about a plan.
+ *   work_total    multiply-adds the plan's rows will perform (sum of w[i])
+ *   class_rows[8] rows per class: 0 empty, 1..5 warp classes (w <= 32, 64, 128, 256, 512),
+ *                 6 block class, 7 large class
+ * Any out-pointer may be NULL.
+ */
+spsyrk_status_t spsyrk_plan_stats(spsyrk_plan_t plan, int64_t *work_total, int64_t class_rows[8]);
+
+/*
+ * spsyrk_plan_buffers - device pointers into the plan's workspace, for inspection and tests:
+ * column pointers colptr[n+1] (int64), the column lists' row ids at_row[nnz] (int32) and
+ * values at_val[nnz] (plan dtype), and the per-row work w[rows] (int64).  Any may be NULL.
+ */
+spsyrk_status_t spsyrk_plan_buffers(spsyrk_plan_t plan, const int64_t **d_colptr, const int32_t **d_at_row,
+                                    const void **d_at_val, const int64_t **d_work);
+
+void spsyrk_destroy(spsyrk_plan_t plan);
+
+const char *spsyrk_status_string(spsyrk_status_t s);
+
+/*
+ * spsyrk_host_tril - the whole path on HOST buffers: copies A to the device, runs plan,
+ * symbolic and numeric, and copies C_L back.  Two calls:
+ *   1. h_c_colidx == NULL: runs plan + symbolic, writes h_c_rowptr[m+1] and *nnz_out, keeps the
+ *      device state in *session.
+ *   2. with h_c_colidx / h_c_vals of *nnz_out entries: runs numeric, copies the result back and
+ *      frees the session.
+ * Device memory for this entry point is allocated and freed by the library (cudaMalloc).
+ * Host buffers should be pinned for full copy speed.  Synchronous.
+ */
+typedef struct spsyrk_session_s *spsyrk_session_t;
+spsyrk_status_t spsyrk_host_tril(spsyrk_session_t *session, int64_t m, int64_t n, int64_t nnz,
+                                 const int64_t *h_rowptr, const int32_t *h_colidx, const void *h_vals,
+                                 spsyrk_dtype_t dtype, spsyrk_mode_t mode,
+                                 int64_t *h_c_rowptr, int64_t *nnz_out,
+                                 int32_t *h_c_colidx, void *h_c_vals);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPSYRK_H */

@@ -1,0 +1,259 @@
+"""ctypes binding of libspsyrk.so: argument marshalling only.
+
+Every function mirrors a C entry point of ``include/spsyrk.h`` under the same name and takes
+torch CUDA tensors (device memory and streams are PyTorch's; the arithmetic is all in the
+library's kernels).  Importing this module loads the CUDA library and raises if it is missing:
+there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspsyrk.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2608_09713_b200.build` "
+        "(nvcc, sm_100a).  The library has no CPU fallback.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK = 0
+F64, F32, I32 = 0, 1, 2
+TRIL, FULL = 0, 1
+NCLASS = 8
+
+_DTYPE_CODE = {torch.float64: F64, torch.float32: F32, torch.int32: I32}
+_CODE_DTYPE = {v: k for k, v in _DTYPE_CODE.items()}
+
+_i64, _vp, _int = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+_szp = ctypes.POINTER(ctypes.c_size_t)
+_i64p = ctypes.POINTER(ctypes.c_int64)
+
+_lib.spsyrk_plan.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _vp, _vp, _int, _int, _i64, _i64, _vp, _szp, _vp]
+_lib.spsyrk_plan_set_rows.argtypes = [_vp, _i64, _i64, _vp]
+_lib.spsyrk_symbolic.argtypes = [_vp, _vp, _i64p, _vp]
+_lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
+_lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
+_lib.spsyrk_jaccard.argtypes = [_i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.spsyrk_plan_stats.argtypes = [_vp, _i64p, _i64p]
+_lib.spsyrk_plan_buffers.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]
+_lib.spsyrk_destroy.argtypes = [_vp]
+_lib.spsyrk_destroy.restype = None
+_lib.spsyrk_status_string.argtypes = [_int]
+_lib.spsyrk_status_string.restype = ctypes.c_char_p
+_lib.spsyrk_host_tril.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _vp, _vp, _int, _int, _vp, _i64p, _vp, _vp]
+for _name in ("spsyrk_plan", "spsyrk_plan_set_rows", "spsyrk_symbolic", "spsyrk_numeric", "spsyrk_mirror",
+              "spsyrk_jaccard", "spsyrk_plan_stats", "spsyrk_plan_buffers", "spsyrk_host_tril"):
+    getattr(_lib, _name).restype = _int
+
+
+class SpsyrkError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {spsyrk_status_string(status)} (status {status})")
+
+
+def spsyrk_status_string(status: int) -> str:
+    return _lib.spsyrk_status_string(status).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise SpsyrkError(status, where)
+
+
+def _p(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dev_check(*tensors):
+    for t in tensors:
+        if t is not None and not (t.is_cuda and t.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    # torch's caching allocator returns 512-byte aligned blocks
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+class Plan:
+    """Owner of a spsyrk_plan_t and of the tensors it borrows (A and the workspace)."""
+
+    def __init__(self, handle, keep, m, n, dtype, mode):
+        self._h, self._keep = handle, keep
+        self.m, self.n, self.dtype, self.mode = m, n, dtype, mode
+        self.row_begin, self.row_end = keep["rows"]
+
+    @property
+    def rows(self):
+        return self.row_end - self.row_begin
+
+    def close(self):
+        if self._h is not None:
+            _lib.spsyrk_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+
+def spsyrk_plan_workspace_bytes(m, n, nnz, dtype=torch.float64, mode=TRIL) -> int:
+    sz = ctypes.c_size_t(0)
+    _check(_lib.spsyrk_plan(None, m, n, nnz, None, None, None, _DTYPE_CODE[dtype], mode, 0, m, None,
+                            ctypes.byref(sz), None), "spsyrk_plan(size query)")
+    return sz.value
+
+
+def spsyrk_plan(m, n, rowptr, colidx, vals, mode=TRIL, row_begin=0, row_end=None, stream=None) -> Plan:
+    _dev_check(rowptr, colidx, vals)
+    assert rowptr.dtype == torch.int64 and colidx.dtype == torch.int32 and vals.dtype in _DTYPE_CODE
+    row_end = m if row_end is None else row_end
+    nnz = colidx.numel()
+    code = _DTYPE_CODE[vals.dtype]
+    sz = ctypes.c_size_t(0)
+    _check(_lib.spsyrk_plan(None, m, n, nnz, None, None, None, code, mode, row_begin, row_end, None,
+                            ctypes.byref(sz), None), "spsyrk_plan(size query)")
+    ws = _workspace(sz.value, rowptr.device)
+    h = _vp()
+    _check(_lib.spsyrk_plan(ctypes.byref(h), m, n, nnz, _p(rowptr), _p(colidx), _p(vals), code, mode, row_begin,
+                            row_end, _p(ws), ctypes.byref(sz), _stream(stream)), "spsyrk_plan")
+    return Plan(h, {"a": (rowptr, colidx, vals), "ws": ws, "rows": (row_begin, row_end)}, m, n, vals.dtype, mode)
+
+
+def spsyrk_plan_set_rows(plan: Plan, row_begin: int, row_end: int, stream=None):
+    _check(_lib.spsyrk_plan_set_rows(plan._h, row_begin, row_end, _stream(stream)), "spsyrk_plan_set_rows")
+    plan.row_begin, plan.row_end = row_begin, row_end
+
+
+def spsyrk_symbolic(plan: Plan, c_rowptr: torch.Tensor, stream=None) -> int:
+    _dev_check(c_rowptr)
+    assert c_rowptr.dtype == torch.int64 and c_rowptr.numel() >= plan.rows + 1
+    nnz = ctypes.c_int64(0)
+    _check(_lib.spsyrk_symbolic(plan._h, _p(c_rowptr), ctypes.byref(nnz), _stream(stream)), "spsyrk_symbolic")
+    return nnz.value
+
+
+def spsyrk_numeric(plan: Plan, c_rowptr, c_colidx, c_vals, stream=None):
+    _dev_check(c_rowptr, c_colidx, c_vals)
+    assert c_colidx.dtype == torch.int32 and c_vals.dtype == plan.dtype
+    _check(_lib.spsyrk_numeric(plan._h, _p(c_rowptr), _p(c_colidx), _p(c_vals), _stream(stream)), "spsyrk_numeric")
+
+
+def spsyrk_destroy(plan: Plan):
+    plan.close()
+
+
+def spsyrk_plan_stats(plan: Plan):
+    work = ctypes.c_int64(0)
+    cls = (ctypes.c_int64 * NCLASS)()
+    _check(_lib.spsyrk_plan_stats(plan._h, ctypes.byref(work), cls), "spsyrk_plan_stats")
+    return work.value, list(cls)
+
+
+def spsyrk_plan_buffers(plan: Plan):
+    """Copies of the plan's column lists and work estimate as torch tensors: (colptr, at_row, at_val, work)."""
+    ptrs = [_vp() for _ in range(4)]
+    _check(_lib.spsyrk_plan_buffers(plan._h, *[ctypes.byref(p) for p in ptrs]), "spsyrk_plan_buffers")
+    nnz = plan._keep["a"][1].numel()
+    dev = plan._keep["a"][0].device
+
+    def view(ptr, count, dtype):
+        if count == 0:
+            return torch.empty(0, dtype=dtype, device=dev)
+        return torch.as_tensor(_DevArray(ptr.value, count, _TYPESTR[dtype]), device=dev).clone()
+
+    torch.cuda.synchronize()
+    return (view(ptrs[0], plan.n + 1, torch.int64), view(ptrs[1], nnz, torch.int32),
+            view(ptrs[2], nnz, plan.dtype), view(ptrs[3], plan.rows, torch.int64))
+
+
+_TYPESTR = {torch.int64: "<i8", torch.int32: "<i4", torch.float64: "<f8", torch.float32: "<f4"}
+
+
+class _DevArray:
+    """A device pointer dressed as a CUDA array so that torch can wrap it without copying."""
+
+    def __init__(self, ptr, count, typestr):
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (ptr, True), "version": 2}
+
+
+def spsyrk_mirror_workspace_bytes(m, nnz_l, dtype) -> int:
+    sz = ctypes.c_size_t(0)
+    _check(_lib.spsyrk_mirror(m, nnz_l, _DTYPE_CODE[dtype], None, None, None, None, None, None, None, None,
+                              ctypes.byref(sz), None), "spsyrk_mirror(size query)")
+    return sz.value
+
+
+def spsyrk_mirror(m, l_rowptr, l_colidx, l_vals, stream=None, workspace=None):
+    """Returns (f_rowptr, f_colidx, f_vals) of F = C_L + C_L^T - D; allocates the outputs with torch."""
+    _dev_check(l_rowptr, l_colidx, l_vals)
+    nnz_l = l_colidx.numel()
+    code = _DTYPE_CODE[l_vals.dtype]
+    sz = ctypes.c_size_t(spsyrk_mirror_workspace_bytes(m, nnz_l, l_vals.dtype))
+    ws = workspace if workspace is not None else _workspace(sz.value, l_rowptr.device)
+    assert ws.numel() >= sz.value
+    sz = ctypes.c_size_t(ws.numel())
+    f_rowptr = torch.empty(m + 1, dtype=torch.int64, device=l_rowptr.device)
+    nnz = ctypes.c_int64(0)
+    st = _stream(stream)
+    _check(_lib.spsyrk_mirror(m, nnz_l, code, _p(l_rowptr), _p(l_colidx), _p(l_vals), _p(f_rowptr), None, None,
+                              ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_mirror(sizes)")
+    f_colidx = torch.empty(max(nnz.value, 1), dtype=torch.int32, device=l_rowptr.device)
+    f_vals = torch.empty(max(nnz.value, 1), dtype=l_vals.dtype, device=l_rowptr.device)
+    _check(_lib.spsyrk_mirror(m, nnz_l, code, _p(l_rowptr), _p(l_colidx), _p(l_vals), _p(f_rowptr), _p(f_colidx),
+                              _p(f_vals), ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_mirror(fill)")
+    return f_rowptr, f_colidx[:nnz.value], f_vals[:nnz.value]
+
+
+def spsyrk_jaccard(m, row_begin, rows, a_rowptr, c_rowptr, c_colidx, c_counts, out=None, stream=None):
+    _dev_check(a_rowptr, c_rowptr, c_colidx, c_counts, out)
+    assert c_counts.dtype == torch.int32
+    if out is None:
+        out = torch.empty(c_counts.numel(), dtype=torch.float32, device=c_counts.device)
+    _check(_lib.spsyrk_jaccard(m, row_begin, rows, _p(a_rowptr), _p(c_rowptr), _p(c_colidx), _p(c_counts), _p(out),
+                               _stream(stream)), "spsyrk_jaccard")
+    return out
+
+
+def spsyrk_host_tril(m, n, rowptr, colidx, vals, mode=TRIL, pinned=True):
+    """Whole path on HOST tensors through the host-buffer entry point.  Returns host tensors
+    (c_rowptr, c_colidx, c_vals); the result buffers are pinned when `pinned`."""
+    assert not rowptr.is_cuda and not colidx.is_cuda and not vals.is_cuda
+    code = _DTYPE_CODE[vals.dtype]
+    nnz = colidx.numel()
+    sess = _vp()
+    c_rowptr = torch.empty(m + 1, dtype=torch.int64, pin_memory=pinned)
+    nnz_c = ctypes.c_int64(0)
+    _check(_lib.spsyrk_host_tril(ctypes.byref(sess), m, n, nnz, _p(rowptr), _p(colidx), _p(vals), code, mode,
+                                 _p(c_rowptr), ctypes.byref(nnz_c), None, None), "spsyrk_host_tril(symbolic)")
+    c_colidx = torch.empty(max(nnz_c.value, 1), dtype=torch.int32, pin_memory=pinned)
+    c_vals = torch.empty(max(nnz_c.value, 1), dtype=vals.dtype, pin_memory=pinned)
+    _check(_lib.spsyrk_host_tril(ctypes.byref(sess), m, n, nnz, None, None, None, code, mode, None, None,
+                                 _p(c_colidx), _p(c_vals)), "spsyrk_host_tril(numeric)")
+    return c_rowptr, c_colidx[:nnz_c.value], c_vals[:nnz_c.value]
+
+
+# ------------------------------------------------------------------------------------------
+# Convenience: the calls a user makes for one product, outputs allocated with torch.
+# ------------------------------------------------------------------------------------------
+def tril_syrk(m, n, rowptr, colidx, vals, mode=TRIL, row_begin=0, row_end=None, plan: Plan | None = None, stream=None):
+    """plan -> symbolic -> numeric.  Returns (c_rowptr, c_colidx, c_vals, plan)."""
+    if plan is None:
+        plan = spsyrk_plan(m, n, rowptr, colidx, vals, mode, row_begin, row_end, stream)
+    c_rowptr = torch.empty(plan.rows + 1, dtype=torch.int64, device=rowptr.device)
+    nnz = spsyrk_symbolic(plan, c_rowptr, stream)
+    c_colidx = torch.empty(max(nnz, 1), dtype=torch.int32, device=rowptr.device)
+    c_vals = torch.empty(max(nnz, 1), dtype=vals.dtype, device=rowptr.device)
+    spsyrk_numeric(plan, c_rowptr, c_colidx, c_vals, stream)
+    return c_rowptr, c_colidx[:nnz], c_vals[:nnz], plan

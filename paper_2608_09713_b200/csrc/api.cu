@@ -1,0 +1,416 @@
+// C ABI: spsyrk_plan / spsyrk_plan_set_rows / spsyrk_symbolic / spsyrk_numeric and helpers.
+// Host-side orchestration only; every step of the path runs in the kernels of the .cuh files.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "rows_cta.cuh"
+#include "rows_warp.cuh"
+
+using namespace spsyrk;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+constexpr int64_t BLOCK_CLASS_MAX_WORK = 16384;  // class 6 (256-thread CTA) up to here, class 7 above
+constexpr uint32_t ROW_CHUNK_BITS_MAX_NUMERIC = 1u << 18;
+constexpr uint32_t ROW_CHUNK_BITS_MAX_SYMBOLIC = 1u << 20;
+constexpr uint32_t COL_CHUNK_BITS_MAX = 1u << 19;
+constexpr size_t LARGE_SMEM_BUDGET = 200 * 1024;
+constexpr uint32_t BLOCK_ACC_SLOTS = 4096;
+
+size_t dtype_size(spsyrk_dtype_t t) { return t == SPSYRK_F64 ? 8 : 4; }
+
+struct Carver {
+    char* base;
+    size_t off = 0;
+    explicit Carver(void* b) : base(static_cast<char*>(b)) {}
+    template <typename T>
+    T* take(size_t count) {
+        off = (off + ALIGN - 1) / ALIGN * ALIGN;
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += count * sizeof(T);
+        return p;
+    }
+};
+
+uint32_t pow2_at_least(uint64_t v, uint32_t lo, uint32_t hi) {
+    uint32_t p = lo;
+    while (p < hi && p < v) p <<= 1;
+    return p;
+}
+
+}  // namespace
+
+struct spsyrk_plan_s {
+    PlanDev dev;
+    spsyrk_dtype_t dtype;
+    int64_t rows_cap;
+    // workspace views
+    int32_t* perm;
+    int32_t* cnt;
+    uint8_t* cls;
+    uint64_t* keys;
+    uint32_t* colcnt;
+    uint32_t* cursor;
+    int32_t* colperm;
+    int32_t* blockhist;
+    int64_t* offsets;
+    int64_t* partials;
+    int64_t* class_start_dev;  // NCLASS + 1
+    unsigned long long* work_total_dev;
+    // host facts
+    int64_t class_start[NCLASS + 1];
+    int64_t work_total;
+    bool have_symbolic;
+    bool key64;
+};
+
+namespace {
+
+size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, size_t sv) {
+    Carver c(ws);
+    const int64_t items = std::max<int64_t>(std::max(m, n), 1);
+    const int64_t nb = bin_blocks(items);
+    auto colptr = c.take<int64_t>(n + 1);
+    auto at_row = c.take<int32_t>(nnz);
+    auto at_val = c.take<char>(nnz * sv);
+    auto desc = c.take<uint2>(nnz);
+    auto work = c.take<int64_t>(m);
+    auto perm = c.take<int32_t>(m);
+    auto cnt = c.take<int32_t>(m);
+    auto cls = c.take<uint8_t>(items);
+    auto keys = c.take<uint64_t>(nnz);
+    auto colcnt = c.take<uint32_t>(n);
+    auto cursor = c.take<uint32_t>(n);
+    auto colperm = c.take<int32_t>(n);
+    auto blockhist = c.take<int32_t>(NCLASS * nb);
+    auto offsets = c.take<int64_t>(NCLASS * nb + 1);
+    auto partials = c.take<int64_t>(scan_partials_count(std::max<int64_t>(items + 1, NCLASS * nb)));
+    auto class_start_dev = c.take<int64_t>(NCLASS + 1);
+    auto work_total_dev = c.take<unsigned long long>(1);
+    auto err = c.take<uint32_t>(1);
+    if (pl) {
+        pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.desc = desc;
+        pl->dev.work = work; pl->dev.err = err;
+        pl->perm = perm; pl->cnt = cnt; pl->cls = cls; pl->keys = keys; pl->colcnt = colcnt; pl->cursor = cursor;
+        pl->colperm = colperm; pl->blockhist = blockhist; pl->offsets = offsets; pl->partials = partials;
+        pl->class_start_dev = class_start_dev; pl->work_total_dev = work_total_dev;
+    }
+    return (c.off + ALIGN - 1) / ALIGN * ALIGN;
+}
+
+spsyrk_status_t read_err(spsyrk_plan_s* pl, cudaStream_t st) {
+    uint32_t e = 0;
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(&e, pl->dev.err, sizeof(e), cudaMemcpyDeviceToHost, st));
+    SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
+    if (e & (ERRW_BAD_ROWPTR | ERRW_BAD_COL | ERRW_UNSORTED)) return SPSYRK_ERR_BAD_CSR;
+    if (e) return SPSYRK_ERR_INTERNAL;
+    return SPSYRK_OK;
+}
+
+template <int G>
+void launch_fill(spsyrk_plan_s* pl, cudaStream_t st) {
+    const PlanDev& P = pl->dev;
+    const int64_t threads = (int64_t)P.m * G;
+    column_fill_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P.rowptr, P.colidx, P.m, P.n, P.colptr,
+                                                                             pl->cursor, pl->keys, P.err);
+}
+
+template <int G>
+void launch_row_work(spsyrk_plan_s* pl, cudaStream_t st) {
+    const PlanDev& P = pl->dev;
+    const int64_t threads = (int64_t)(P.r1 - P.r0) * G;
+    row_work_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P, pl->cls, BLOCK_CLASS_MAX_WORK, pl->work_total_dev);
+}
+
+int group_width(int64_t nnz, int64_t m) {
+    const double avg = m > 0 ? (double)nnz / (double)m : 0.0;
+    return avg <= 4 ? 4 : avg <= 8 ? 8 : avg <= 16 ? 16 : 32;
+}
+
+template <typename V, int R, int G>
+void launch_colsort_group(spsyrk_plan_s* pl, int64_t first, int64_t count, cudaStream_t st) {
+    if (count <= 0) return;
+    const int64_t threads = count * G;
+    column_sort_group_kernel<V, R, G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(pl->dev, pl->colperm + first, count, pl->keys);
+}
+
+template <typename V>
+spsyrk_status_t sort_columns(spsyrk_plan_s* pl, const int64_t* cs, cudaStream_t st) {
+    launch_colsort_group<V, 1, 8>(pl, cs[1], cs[2] - cs[1], st);
+    launch_colsort_group<V, 1, 16>(pl, cs[2], cs[3] - cs[2], st);
+    launch_colsort_group<V, 1, 32>(pl, cs[3], cs[4] - cs[3], st);
+    launch_colsort_group<V, 2, 32>(pl, cs[4], cs[5] - cs[4], st);
+    launch_colsort_group<V, 4, 32>(pl, cs[5], cs[6] - cs[5], st);
+    launch_colsort_group<V, 8, 32>(pl, cs[6], cs[7] - cs[6], st);
+    const int64_t big = cs[8] - cs[7];
+    if (big > 0) {
+        const uint32_t cb = pow2_at_least((uint64_t)pl->dev.m, 1024u, COL_CHUNK_BITS_MAX);
+        const size_t smem = (size_t)(cb >> 5) * 2 * sizeof(uint32_t);
+        SPSYRK_CUDA_TRY(cudaFuncSetAttribute(column_sort_cta_kernel<V, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        column_sort_cta_kernel<V, 512><<<(unsigned)big, 512, smem, st>>>(pl->dev, pl->colperm + cs[7], pl->keys, cb);
+    }
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    return SPSYRK_OK;
+}
+
+// work estimate + binning of the plan's current row range; reads class sizes back (one sync)
+spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
+    const PlanDev& P = pl->dev;
+    const int64_t rows = P.r1 - P.r0;
+    pl->have_symbolic = false;
+    SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->work_total_dev, 0, sizeof(unsigned long long), st));
+    if (rows > 0) {
+        switch (group_width(P.nnz, P.m)) {
+            case 4: launch_row_work<4>(pl, st); break;
+            case 8: launch_row_work<8>(pl, st); break;
+            case 16: launch_row_work<16>(pl, st); break;
+            default: launch_row_work<32>(pl, st); break;
+        }
+    }
+    SPSYRK_CUDA_TRY(bin_items(pl->cls, rows, pl->perm, pl->class_start_dev, pl->blockhist, pl->offsets, pl->partials, st));
+    unsigned long long wt = 0;
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(pl->class_start, pl->class_start_dev, sizeof(pl->class_start), cudaMemcpyDeviceToHost, st));
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(&wt, pl->work_total_dev, sizeof(wt), cudaMemcpyDeviceToHost, st));
+    spsyrk_status_t s = read_err(pl, st);
+    pl->work_total = (int64_t)wt;
+    return s;
+}
+
+template <int N>
+void launch_symbolic_warp(spsyrk_plan_s* pl, int c, cudaStream_t st) {
+    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    if (count <= 0) return;
+    symbolic_warp_kernel<N><<<(unsigned)((count + ROW_WARPS - 1) / ROW_WARPS), ROW_WARPS * 32, 0, st>>>(
+        pl->dev, pl->perm + pl->class_start[c], count, pl->cnt);
+}
+
+template <typename V, int N, typename Key>
+void launch_numeric_warp(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    if (count <= 0) return;
+    constexpr int NW = numeric_warps(N);
+    numeric_warp_kernel<V, N, Key><<<(unsigned)((count + NW - 1) / NW), NW * 32, 0, st>>>(
+        pl->dev, pl->perm + pl->class_start[c], count, c_rowptr, c_colidx, static_cast<V*>(c_vals));
+}
+
+template <typename V, typename Key>
+void launch_numeric_warp_all(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    launch_numeric_warp<V, 32, Key>(pl, 1, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 64, Key>(pl, 2, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 128, Key>(pl, 3, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 256, Key>(pl, 4, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 512, Key>(pl, 5, c_rowptr, c_colidx, c_vals, st);
+}
+
+uint32_t row_chunk_bits(const spsyrk_plan_s* pl, uint32_t cap) {
+    const uint64_t umax = pl->dev.mode == SPSYRK_TRIL ? (uint64_t)pl->dev.r1 : (uint64_t)pl->dev.m;
+    return pow2_at_least(umax, 1024u, cap);
+}
+
+template <int THREADS>
+spsyrk_status_t launch_symbolic_cta(spsyrk_plan_s* pl, int c, cudaStream_t st) {
+    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    if (count <= 0) return SPSYRK_OK;
+    const uint32_t cb = row_chunk_bits(pl, ROW_CHUNK_BITS_MAX_SYMBOLIC);
+    const size_t smem = CtaRowSmem<int32_t, THREADS, false>::bytes(cb, 0);
+    auto kern = rows_cta_kernel<int32_t, THREADS, false>;
+    SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, 0u, pl->cnt, nullptr, nullptr, nullptr);
+    return SPSYRK_OK;
+}
+
+template <typename V, int THREADS>
+spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_or_zero, const int64_t* c_rowptr, int32_t* c_colidx,
+                                   void* c_vals, cudaStream_t st) {
+    using Acc = typename AccOf<V>::type;
+    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    if (count <= 0) return SPSYRK_OK;
+    const uint32_t cb = row_chunk_bits(pl, ROW_CHUNK_BITS_MAX_NUMERIC);
+    uint32_t slots = acc_slots_or_zero;
+    if (slots == 0) {
+        const size_t fixed = CtaRowSmem<V, THREADS, true>::bytes(cb, 0);
+        slots = (uint32_t)((LARGE_SMEM_BUDGET - fixed) / sizeof(Acc));
+        slots = std::min(slots, cb);  // a chunk never has more slots than bits
+    }
+    const size_t smem = CtaRowSmem<V, THREADS, true>::bytes(cb, slots);
+    auto kern = rows_cta_kernel<V, THREADS, true>;
+    SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, c_rowptr, c_colidx,
+                                                  static_cast<V*>(c_vals));
+    return SPSYRK_OK;
+}
+
+template <typename V>
+spsyrk_status_t numeric_typed(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    if (pl->key64) launch_numeric_warp_all<V, uint64_t>(pl, c_rowptr, c_colidx, c_vals, st);
+    else launch_numeric_warp_all<V, uint32_t>(pl, c_rowptr, c_colidx, c_vals, st);
+    spsyrk_status_t s = launch_numeric_cta<V, 256>(pl, 6, BLOCK_ACC_SLOTS, c_rowptr, c_colidx, c_vals, st);
+    if (s != SPSYRK_OK) return s;
+    s = launch_numeric_cta<V, 1024>(pl, 7, 0u, c_rowptr, c_colidx, c_vals, st);
+    if (s != SPSYRK_OK) return s;
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    return SPSYRK_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t nnz, const int64_t* d_rowptr,
+                            const int32_t* d_colidx, const void* d_vals, spsyrk_dtype_t dtype, spsyrk_mode_t mode,
+                            int64_t row_begin, int64_t row_end, void* d_workspace, size_t* workspace_bytes,
+                            void* cuda_stream) {
+    if (!workspace_bytes || m < 0 || n < 0 || nnz < 0) return SPSYRK_ERR_INVALID_ARG;
+    if (dtype != SPSYRK_F64 && dtype != SPSYRK_F32 && dtype != SPSYRK_I32) return SPSYRK_ERR_INVALID_ARG;
+    if (mode != SPSYRK_TRIL && mode != SPSYRK_FULL) return SPSYRK_ERR_INVALID_ARG;
+    if (row_begin < 0 || row_end < row_begin || row_end > m) return SPSYRK_ERR_INVALID_ARG;
+    if (m >= (int64_t(1) << 31) - 1 || n >= (int64_t(1) << 31) - 1 || nnz >= (int64_t(1) << 31) - 1) return SPSYRK_ERR_OVERFLOW;
+    const size_t sv = dtype_size(dtype);
+    const size_t need = carve(nullptr, nullptr, m, n, nnz, sv);
+    if (!d_workspace) {
+        *workspace_bytes = need;
+        return SPSYRK_OK;
+    }
+    if (!plan || !d_rowptr || (nnz > 0 && (!d_colidx || !d_vals))) return SPSYRK_ERR_INVALID_ARG;
+    if (*workspace_bytes < need) return SPSYRK_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(d_workspace) % ALIGN) return SPSYRK_ERR_INVALID_ARG;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    spsyrk_plan_s* pl = new (std::nothrow) spsyrk_plan_s();
+    if (!pl) return SPSYRK_ERR_INTERNAL;
+    std::memset(pl, 0, sizeof(*pl));
+    PlanDev& P = pl->dev;
+    P.m = (int32_t)m; P.n = (int32_t)n; P.nnz = nnz; P.r0 = (int32_t)row_begin; P.r1 = (int32_t)row_end; P.mode = (int32_t)mode;
+    P.rowptr = d_rowptr; P.colidx = d_colidx; P.vals = d_vals;
+    pl->dtype = dtype;
+    pl->rows_cap = m;
+    pl->key64 = m > (int64_t(1) << 22);
+    carve(pl, d_workspace, m, n, nnz, sv);
+
+    auto fail = [&](spsyrk_status_t s) { delete pl; return s; };
+#define PLAN_TRY(expr) do { if ((expr) != cudaSuccess) return fail(SPSYRK_ERR_CUDA); } while (0)
+    PLAN_TRY(cudaMemsetAsync(P.err, 0, sizeof(uint32_t), st));
+    if (n > 0) {
+        PLAN_TRY(cudaMemsetAsync(pl->colcnt, 0, (size_t)n * sizeof(uint32_t), st));
+        PLAN_TRY(cudaMemsetAsync(pl->cursor, 0, (size_t)n * sizeof(uint32_t), st));
+    }
+    // 1. row pointers must be sane before anything indexes with them
+    validate_rowptr_kernel<<<(unsigned)((m + 1 + 255) / 256), 256, 0, st>>>(d_rowptr, m, nnz, P.err);
+    PLAN_TRY(cudaGetLastError());
+    spsyrk_status_t s = read_err(pl, st);
+    if (s != SPSYRK_OK) return fail(s);
+    // 2. transpose: histogram, scan, keyed scatter, per-column sort
+    if (nnz > 0) {
+        const unsigned hb = (unsigned)std::min<int64_t>((nnz + 255) / 256, 148 * 32);
+        column_histogram_kernel<<<hb, 256, 0, st>>>(d_colidx, nnz, P.n, pl->colcnt, P.err);
+    }
+    PLAN_TRY(exclusive_scan_i64<uint32_t>(pl->colcnt, n, P.colptr, pl->partials, st));
+    if (nnz > 0) {
+        switch (group_width(nnz, m)) {
+            case 4: launch_fill<4>(pl, st); break;
+            case 8: launch_fill<8>(pl, st); break;
+            case 16: launch_fill<16>(pl, st); break;
+            default: launch_fill<32>(pl, st); break;
+        }
+    }
+    if (n > 0) column_class_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(P.colptr, P.n, pl->cls);
+    PLAN_TRY(bin_items(pl->cls, n, pl->colperm, pl->class_start_dev, pl->blockhist, pl->offsets, pl->partials, st));
+    int64_t cs[NCLASS + 1];
+    PLAN_TRY(cudaMemcpyAsync(cs, pl->class_start_dev, sizeof(cs), cudaMemcpyDeviceToHost, st));
+    s = read_err(pl, st);  // synchronises; column ids are known to be in range and rows sorted from here on
+    if (s != SPSYRK_OK) return fail(s);
+    s = sv == 8 ? sort_columns<uint64_t>(pl, cs, st) : sort_columns<uint32_t>(pl, cs, st);
+    if (s != SPSYRK_OK) return fail(s);
+    // 3. work estimate and row binning
+    s = estimate_and_bin(pl, st);
+    if (s != SPSYRK_OK) return fail(s);
+#undef PLAN_TRY
+    *plan = pl;
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_plan_set_rows(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end, void* cuda_stream) {
+    if (!plan || row_begin < 0 || row_end < row_begin || row_end > plan->dev.m) return SPSYRK_ERR_INVALID_ARG;
+    plan->dev.r0 = (int32_t)row_begin;
+    plan->dev.r1 = (int32_t)row_end;
+    return estimate_and_bin(plan, static_cast<cudaStream_t>(cuda_stream));
+}
+
+spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t* d_c_rowptr, int64_t* nnz_out, void* cuda_stream) {
+    if (!plan || !d_c_rowptr || !nnz_out) return SPSYRK_ERR_INVALID_ARG;
+    spsyrk_plan_s* pl = plan;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t rows = pl->dev.r1 - pl->dev.r0;
+    if (rows > 0) SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->cnt, 0, (size_t)rows * sizeof(int32_t), st));
+    launch_symbolic_warp<32>(pl, 1, st);
+    launch_symbolic_warp<64>(pl, 2, st);
+    launch_symbolic_warp<128>(pl, 3, st);
+    launch_symbolic_warp<256>(pl, 4, st);
+    launch_symbolic_warp<512>(pl, 5, st);
+    spsyrk_status_t s = launch_symbolic_cta<256>(pl, 6, st);
+    if (s != SPSYRK_OK) return s;
+    s = launch_symbolic_cta<1024>(pl, 7, st);
+    if (s != SPSYRK_OK) return s;
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<int32_t>(pl->cnt, rows, d_c_rowptr, pl->partials, st));
+    int64_t nnz = 0;
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(&nnz, d_c_rowptr + rows, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
+    s = read_err(pl, st);
+    if (s != SPSYRK_OK) return s;
+    *nnz_out = nnz;
+    pl->have_symbolic = true;
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t* d_c_rowptr, int32_t* d_c_colidx, void* d_c_vals,
+                               void* cuda_stream) {
+    if (!plan || !d_c_rowptr) return SPSYRK_ERR_INVALID_ARG;
+    spsyrk_plan_s* pl = plan;
+    if (!pl->have_symbolic) return SPSYRK_ERR_SEQUENCE;
+    if (pl->work_total > 0 && (!d_c_colidx || !d_c_vals)) return SPSYRK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    switch (pl->dtype) {
+        case SPSYRK_F64: return numeric_typed<double>(pl, d_c_rowptr, d_c_colidx, d_c_vals, st);
+        case SPSYRK_F32: return numeric_typed<float>(pl, d_c_rowptr, d_c_colidx, d_c_vals, st);
+        default: return numeric_typed<int32_t>(pl, d_c_rowptr, d_c_colidx, d_c_vals, st);
+    }
+}
+
+spsyrk_status_t spsyrk_plan_stats(spsyrk_plan_t plan, int64_t* work_total, int64_t class_rows[8]) {
+    if (!plan) return SPSYRK_ERR_INVALID_ARG;
+    if (work_total) *work_total = plan->work_total;
+    if (class_rows)
+        for (int c = 0; c < NCLASS; ++c) class_rows[c] = plan->class_start[c + 1] - plan->class_start[c];
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_plan_buffers(spsyrk_plan_t plan, const int64_t** d_colptr, const int32_t** d_at_row,
+                                    const void** d_at_val, const int64_t** d_work) {
+    if (!plan) return SPSYRK_ERR_INVALID_ARG;
+    if (d_colptr) *d_colptr = plan->dev.colptr;
+    if (d_at_row) *d_at_row = plan->dev.at_row;
+    if (d_at_val) *d_at_val = plan->dev.at_val;
+    if (d_work) *d_work = plan->dev.work;
+    return SPSYRK_OK;
+}
+
+void spsyrk_destroy(spsyrk_plan_t plan) { delete plan; }
+
+const char* spsyrk_status_string(spsyrk_status_t s) {
+    switch (s) {
+        case SPSYRK_OK: return "ok";
+        case SPSYRK_ERR_INVALID_ARG: return "invalid argument";
+        case SPSYRK_ERR_BAD_CSR: return "input is not canonical CSR";
+        case SPSYRK_ERR_WORKSPACE: return "workspace too small";
+        case SPSYRK_ERR_OVERFLOW: return "size exceeds the supported range";
+        case SPSYRK_ERR_SEQUENCE: return "call sequence error";
+        case SPSYRK_ERR_CUDA: return "CUDA runtime error";
+        case SPSYRK_ERR_INTERNAL: return "internal error";
+        case SPSYRK_ERR_NOT_IMPLEMENTED: return "not implemented";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,171 @@
+// Steps a4 / a6 for heavy rows: one CTA per output row.
+//
+// The output columns j of row i lie in [0, U), U = i + 1 (TRIL) or m (FULL).  The range is cut
+// into chunks of `chunk_bits` columns.  For each chunk a shared-memory bitmap records which j
+// occur; a prefix population count over its words turns the bitmap into an order-preserving map
+// j -> output slot (number of set bits below j), so rows come out sorted with no sort at all:
+//   symbolic : the row count is the number of set bits over all chunks;
+//   numeric  : partial products are added into shared-memory accumulators indexed by slot
+//              (tiles of `acc_slots` slots; a tile is a contiguous range of j, found per column
+//              list by binary search, the lists being ascending in j), then tiles are written out
+//              contiguously; column ids are regenerated from the bitmap.
+// Work is spread over the CTA by flattening the (list, position) pairs of up to THREADS lists at
+// a time through a prefix sum of their lengths, so that one very long list is shared by all lanes.
+#pragma once
+#include "transpose.cuh"
+
+namespace spsyrk {
+
+enum : int { CTA_SETBITS = 0, CTA_ACCUM = 1 };
+
+template <typename V, int THREADS, bool NUMERIC>
+struct CtaRowSmem {
+    using Acc = typename AccOf<V>::type;
+    static size_t bytes(uint32_t chunk_bits, uint32_t acc_slots) {
+        size_t words = (size_t)(chunk_bits >> 5) * (NUMERIC ? 2 : 1) + 2 * THREADS + 1;
+        words = (words + 3) & ~size_t(3);
+        size_t b = words * 4;
+        if (NUMERIC) b += (size_t)THREADS * sizeof(Acc) + (size_t)acc_slots * sizeof(Acc);
+        return b;
+    }
+};
+
+template <typename V, int THREADS, bool NUMERIC>
+__global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int32_t* __restrict__ rows,
+                                                           uint32_t chunk_bits, uint32_t acc_slots,
+                                                           int32_t* __restrict__ cnt,
+                                                           const int64_t* __restrict__ c_rowptr,
+                                                           int32_t* __restrict__ c_colidx, V* __restrict__ c_vals) {
+    using Acc = typename AccOf<V>::type;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ uint32_t scratch[33];
+    __shared__ uint32_t s_sel[2];
+    const uint32_t cw = chunk_bits >> 5;
+    uint32_t* bits = reinterpret_cast<uint32_t*>(smem_raw);
+    uint32_t* rank = bits + cw;  // numeric only
+    uint32_t* loff = bits + (size_t)cw * (NUMERIC ? 2 : 1);
+    uint32_t* lstart = loff + THREADS + 1;
+    size_t words = (size_t)cw * (NUMERIC ? 2 : 1) + 2 * THREADS + 1;
+    words = (words + 3) & ~size_t(3);
+    Acc* la = reinterpret_cast<Acc*>(smem_raw + words * 4);
+    Acc* acc = la + THREADS;
+
+    const int tid = threadIdx.x;
+    const int32_t rloc = rows[blockIdx.x];
+    const int64_t i = (int64_t)P.r0 + rloc;
+    const uint32_t U = P.mode == SPSYRK_TRIL ? (uint32_t)i + 1u : (uint32_t)P.m;
+    const int64_t p0 = P.rowptr[i];
+    const uint32_t deg = (uint32_t)(P.rowptr[i + 1] - p0);
+    const int64_t out_base = NUMERIC ? c_rowptr[rloc] : 0;
+    const uint32_t per = (cw + THREADS - 1) / THREADS;
+    const uint32_t w0 = tid * per;
+    uint32_t total_cnt = 0;
+
+    // Visit every partial product whose j lies in [lo, hi); `whole` skips the per-list search.
+    auto for_each_product = [&](auto what, uint32_t lo, uint32_t hi, bool whole, uint32_t c0, uint32_t s0) {
+        constexpr int WHAT = decltype(what)::value;
+        for (uint32_t b0 = 0; b0 < deg; b0 += THREADS) {
+            uint32_t sublen = 0, substart = 0;
+            Acc a = Acc(0);
+            if (b0 + tid < deg) {
+                const uint2 d = P.desc[p0 + b0 + tid];
+                if (whole) {
+                    substart = d.x;
+                    sublen = d.y;
+                } else {
+                    const int32_t* lst = P.at_row + d.x;
+                    const uint32_t a0 = lo == 0 ? 0u : lower_bound_i32(lst, d.y, (int32_t)lo);
+                    const uint32_t a1 = lower_bound_i32(lst, d.y, (int32_t)hi);
+                    substart = d.x + a0;
+                    sublen = a1 - a0;
+                }
+                if (WHAT == CTA_ACCUM) a = (Acc) static_cast<const V*>(P.vals)[p0 + b0 + tid];
+            }
+            uint32_t T;
+            const uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(sublen, scratch, &T);
+            loff[tid] = ex;
+            lstart[tid] = substart;
+            if (WHAT == CTA_ACCUM) la[tid] = a;
+            if (tid == 0) loff[THREADS] = T;
+            __syncthreads();
+            uint32_t cur = 0;
+            for (uint32_t item = tid; item < T; item += THREADS) {
+                while (item >= loff[cur + 1]) ++cur;
+                const uint32_t q = lstart[cur] + (item - loff[cur]);
+                const uint32_t rel = (uint32_t)P.at_row[q] - c0;
+                if (WHAT == CTA_SETBITS) {
+                    atomicOr(&bits[rel >> 5], 1u << (rel & 31));
+                } else {
+                    const uint32_t slot = rank[rel >> 5] + __popc(bits[rel >> 5] & ((1u << (rel & 31)) - 1u)) - s0;
+                    atomicAdd(&acc[slot], acc_mul(la[cur], (Acc) static_cast<const V*>(P.at_val)[q]));
+                }
+            }
+            __syncthreads();
+        }
+    };
+
+    for (uint32_t c0 = 0; c0 < U; c0 += chunk_bits) {
+        const uint32_t c1 = min(c0 + chunk_bits, U);
+        const bool single_chunk = (c0 == 0 && c1 == U);
+        for (uint32_t w = tid; w < cw; w += THREADS) bits[w] = 0;
+        __syncthreads();
+        for_each_product(std::integral_constant<int, CTA_SETBITS>{}, c0, c1, single_chunk, c0, 0u);
+        uint32_t s = 0;
+        for (uint32_t w = w0; w < w0 + per && w < cw; ++w) s += __popc(bits[w]);
+        uint32_t tot;
+        uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(s, scratch, &tot);
+        if (NUMERIC) {
+            for (uint32_t w = w0; w < w0 + per && w < cw; ++w) { rank[w] = ex; ex += __popc(bits[w]); }
+            __syncthreads();
+            const int64_t ob = out_base + total_cnt;
+            // column ids straight from the bitmap
+            for (uint32_t w = tid; w < cw; w += THREADS) {
+                uint32_t b = bits[w], r = rank[w];
+                while (b) {
+                    const int bit = __ffs(b) - 1;
+                    c_colidx[ob + r] = (int32_t)(c0 + (w << 5) + bit);
+                    ++r;
+                    b &= b - 1;
+                }
+            }
+            for (uint32_t s0 = 0; s0 < tot; s0 += acc_slots) {
+                const uint32_t s1 = min(s0 + acc_slots, tot);
+                const bool single_tile = (s0 == 0 && s1 == tot);
+                uint32_t jlo = c0, jhi = c1;
+                if (!single_tile) {
+                    if (tid < 2) {
+                        const uint32_t sl = tid == 0 ? s0 : s1;
+                        uint32_t res;
+                        if (tid == 0 && s0 == 0) res = c0;
+                        else if (tid == 1 && s1 == tot) res = c1;
+                        else {
+                            // last word whose rank is <= sl holds slot sl
+                            uint32_t lo_w = 0, hi_w = cw;
+                            while (hi_w - lo_w > 1) {
+                                uint32_t mid = (lo_w + hi_w) >> 1;
+                                if (rank[mid] <= sl) lo_w = mid; else hi_w = mid;
+                            }
+                            uint32_t b = bits[lo_w];
+                            for (uint32_t n = sl - rank[lo_w]; n > 0; --n) b &= b - 1;
+                            res = c0 + (lo_w << 5) + (uint32_t)(__ffs(b) - 1);
+                        }
+                        s_sel[tid] = res;
+                    }
+                    __syncthreads();
+                    jlo = s_sel[0];
+                    jhi = s_sel[1];
+                }
+                for (uint32_t t = tid; t < s1 - s0; t += THREADS) acc[t] = Acc(0);
+                __syncthreads();
+                for_each_product(std::integral_constant<int, CTA_ACCUM>{}, jlo, jhi, single_chunk && single_tile, c0, s0);
+                for (uint32_t t = tid; t < s1 - s0; t += THREADS) c_vals[ob + s0 + t] = (V)acc[t];
+                __syncthreads();
+            }
+        }
+        total_cnt += tot;
+        __syncthreads();
+    }
+    if (!NUMERIC && tid == 0) cnt[rloc] = (int32_t)total_cnt;
+}
+
+}  // namespace spsyrk

@@ -1,0 +1,241 @@
+"""Parity of the CUDA path against the CPU oracle, element by element, through the C ABI.
+
+Bars: CSR structure and int32 values bit-exact; fp64 values within 1e-12 and fp32 values within
+1e-5 of the oracle relative to the sum of absolute partial products of the entry (which equals
+the relative error whenever the partial products share a sign); Jaccard within 1e-5.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_09713_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TOL = {np.dtype(np.float64): 1e-12, np.dtype(np.float32): 1e-5}
+
+
+@pytest.fixture(scope="module")
+def B():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    from paper_2608_09713_b200 import binding
+    return binding
+
+
+def dev(a: W.CSR):
+    return (torch.from_numpy(a.rowptr).cuda(), torch.from_numpy(a.colidx).cuda(), torch.from_numpy(a.vals).cuda())
+
+
+def check_values(gpu_vals, ref, dtype):
+    """gpu_vals: numpy array of the matrix dtype; ref: oracle SyrkResult-like (vals, absvals float64)."""
+    if np.issubdtype(dtype, np.integer):
+        assert np.array_equal(gpu_vals, oracle.to_int32(ref.vals))
+        return 0.0
+    err = np.abs(gpu_vals.astype(np.float64) - ref.vals)
+    bound = TOL[np.dtype(dtype)] * ref.absvals
+    assert np.all(err <= bound), f"max scaled error {np.max(err / np.maximum(ref.absvals, 1e-300)):.3e}"
+    return float(np.max(err / np.maximum(ref.absvals, 1e-300))) if err.size else 0.0
+
+
+def run_and_compare(B, a: W.CSR, mode, r0=0, r1=None, cols=None, plan=None):
+    r1 = a.m if r1 is None else r1
+    d = dev(a)
+    c_rowptr, c_colidx, c_vals, plan = B.tril_syrk(a.m, a.n, *d, mode=mode, row_begin=r0, row_end=r1, plan=plan)
+    torch.cuda.synchronize()
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, mode, r0, r1, cols=cols)
+    assert np.array_equal(c_rowptr.cpu().numpy(), ref.rowptr)
+    assert np.array_equal(c_colidx.cpu().numpy(), ref.colidx)
+    check_values(c_vals.cpu().numpy(), ref, a.vals.dtype)
+    work, classes = B.spsyrk_plan_stats(plan)
+    assert work == int(ref.work.sum())
+    assert sum(classes) == r1 - r0
+    return (c_rowptr, c_colidx, c_vals), ref, plan
+
+
+# ------------------------------------------------------------------ the five workloads, reduced
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_small_configs(B, idx, mode):
+    a = W.small(idx)
+    run_and_compare(B, a, mode)
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_plan_internals(B, idx):
+    """Step a1 (column lists ascending by row) and step a2 (per-row work) against the oracle."""
+    a = W.small(idx)
+    plan = B.spsyrk_plan(a.m, a.n, *dev(a))
+    colptr, at_row, at_val, work = (t.cpu().numpy() for t in B.spsyrk_plan_buffers(plan))
+    cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
+    assert np.array_equal(colptr, cols.colptr)
+    assert np.array_equal(at_row, cols.rows)
+    assert np.array_equal(at_val.astype(np.float64), cols.vals)
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, cols=cols, counts_only=True)
+    assert np.array_equal(work, ref.work)
+    d = np.diff(cols.colptr)
+    total, classes = B.spsyrk_plan_stats(plan)
+    assert total == int((d * (d + 1) // 2).sum())           # closed form of the multiply-add count
+    fplan = B.spsyrk_plan(a.m, a.n, *dev(a), mode=B.FULL)
+    assert B.spsyrk_plan_stats(fplan)[0] == int((d * d).sum())
+
+
+def test_rmat_unpermuted_and_row_classes(B):
+    """Hubs at low indices; every row class must be populated somewhere in these cases."""
+    seen = np.zeros(8, dtype=np.int64)
+    for a in (W.rmat(13, 16, 21, permute=False), W.small(3), W.small(2), W.small(5)):
+        _, _, plan = run_and_compare(B, a, 0)
+        seen += np.array(B.spsyrk_plan_stats(plan)[1])
+    assert (seen > 0).all(), f"row classes not all exercised: {seen}"
+
+
+@pytest.mark.parametrize("idx", [2, 3, 5])
+def test_row_tiles_concatenate(B, idx):
+    a = W.small(idx)
+    cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
+    full, ref, _ = run_and_compare(B, a, 0, cols=cols)
+    cuts = [0, a.m // 7, a.m // 7 + 1, a.m // 2, a.m - 3, a.m]
+    plan = None
+    parts_col, parts_val, counts = [], [], []
+    for r0, r1 in zip(cuts[:-1], cuts[1:]):
+        if plan is not None:
+            B.spsyrk_plan_set_rows(plan, r0, r1)        # re-target without repeating the transpose
+        (rp, ci, cv), _, plan = run_and_compare(B, a, 0, r0, r1, cols=cols, plan=plan)
+        parts_col.append(ci); parts_val.append(cv); counts.append(rp[1:] - rp[:-1])
+    assert torch.equal(torch.cat(counts), full[0][1:] - full[0][:-1])
+    assert torch.equal(torch.cat(parts_col), full[1])
+    assert torch.equal(torch.cat(parts_val), full[2])   # deterministic row classes give identical bits
+
+
+def test_warp_rows_are_bit_reproducible_and_match_oracle_order(B):
+    """Light rows sum partial products in ascending k like the oracle: fp64 results are identical bits."""
+    a = W.small(5)
+    (_, _, v1), ref, _ = run_and_compare(B, a, 0)
+    (_, _, v2), _, _ = run_and_compare(B, a, 0)
+    assert torch.equal(v1, v2)
+    assert np.array_equal(v1.cpu().numpy(), ref.vals)
+
+
+# ------------------------------------------------------------------------------ edge cases
+def _csr(dense):
+    dense = np.asarray(dense, dtype=np.float64)
+    m, n = dense.shape
+    s = dense != 0
+    rowptr = np.zeros(m + 1, dtype=np.int64)
+    np.cumsum(s.sum(axis=1), out=rowptr[1:])
+    rr, cc = np.nonzero(s)
+    return W.CSR(m, n, rowptr, cc.astype(np.int32), dense[rr, cc].copy())
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_edge_cases(B, mode):
+    rng = np.random.default_rng(4)
+    cases = []
+    cases.append(_csr(np.zeros((5, 4))))                                          # nnz = 0
+    cases.append(_csr(np.array([[2.0, 0.0, 3.0]])))                               # m = 1
+    cases.append(_csr(np.array([[2.0], [0.0], [5.0], [1.0]])))                    # n = 1
+    d = (rng.random((40, 30)) < 0.2) * rng.random((40, 30)); d[3] = 0; d[17] = 0; d[:, 5] = 0
+    cases.append(_csr(d))                                                         # empty rows and column
+    d = (rng.random((70, 50)) < 0.1) * rng.random((70, 50)); d[9] = rng.random(50) + 0.1
+    cases.append(_csr(d))                                                         # a full row (more than 32 nonzeros)
+    d = (rng.random((300, 40)) < 0.05) * rng.random((300, 40)); d[:, 7] = rng.random(300) + 0.1
+    cases.append(_csr(d))                                                         # a full column: dense output
+    d = (rng.random((64, 64)) < 0.3) * rng.random((64, 64)); d[40] = d[2]; d[63] = d[2]
+    cases.append(_csr(d))                                                         # identical rows
+    cases.append(_csr(rng.random((90, 70)) + 0.1))                                # fully dense A
+    for a in cases:
+        run_and_compare(B, a, mode)
+
+
+def test_zero_rows(B):
+    a = W.CSR(0, 5, np.zeros(1, dtype=np.int64), np.zeros(0, dtype=np.int32), np.zeros(0, dtype=np.float64))
+    rp, ci, cv, plan = B.tril_syrk(0, 5, *dev(a))
+    assert rp.cpu().tolist() == [0] and ci.numel() == 0
+
+
+def test_cancellation_keeps_structural_entries(B):
+    d = np.array([[1.0, 1.0, 0.0], [1.0, -1.0, 0.0], [0.0, 0.0, 2.0]])
+    rp, ci, cv, _ = B.tril_syrk(3, 3, *dev(_csr(d)))
+    assert rp.cpu().tolist() == [0, 1, 3, 4] and ci.cpu().tolist() == [0, 0, 1, 2]
+    assert cv.cpu().tolist() == [2.0, 0.0, 2.0, 4.0]
+
+
+def test_bad_csr_is_rejected(B):
+    a = W.small(1)
+    rowptr, colidx, vals = dev(a)
+    bad = colidx.clone(); bad[3], bad[4] = colidx[4].item(), colidx[3].item()       # unsorted row
+    with pytest.raises(B.SpsyrkError) as e:
+        B.spsyrk_plan(a.m, a.n, rowptr, bad, vals)
+    assert e.value.status == 2
+    bad = colidx.clone(); bad[10] = a.n                                               # out of range
+    with pytest.raises(B.SpsyrkError) as e:
+        B.spsyrk_plan(a.m, a.n, rowptr, bad, vals)
+    assert e.value.status == 2
+    bad = colidx.clone(); bad[1] = bad[0]                                             # duplicate
+    with pytest.raises(B.SpsyrkError) as e:
+        B.spsyrk_plan(a.m, a.n, rowptr, bad, vals)
+    assert e.value.status == 2
+    badp = rowptr.clone(); badp[5] = badp[6] + 1                                      # non-monotone
+    with pytest.raises(B.SpsyrkError) as e:
+        B.spsyrk_plan(a.m, a.n, badp, colidx, vals)
+    assert e.value.status == 2
+    plan = B.spsyrk_plan(a.m, a.n, rowptr, colidx, vals)
+    with pytest.raises(B.SpsyrkError) as e:                                           # numeric before symbolic
+        B.spsyrk_numeric(plan, torch.zeros(a.m + 1, dtype=torch.int64, device="cuda"),
+                         torch.zeros(1, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.float64, device="cuda"))
+    assert e.value.status == 5
+
+
+# ----------------------------------------------------------------------------------- mirror
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_mirror(B, idx):
+    a = W.small(idx)
+    (rp, ci, cv), ref, _ = run_and_compare(B, a, 0)
+    f_rowptr, f_colidx, f_vals = B.spsyrk_mirror(a.m, rp, ci, cv)
+    torch.cuda.synchronize()
+    lv = cv.cpu().numpy()
+    o_rowptr, o_colidx, o_vals = oracle.mirror(a.m, rp.cpu().numpy(), ci.cpu().numpy(), lv.astype(np.float64))
+    assert np.array_equal(f_rowptr.cpu().numpy(), o_rowptr)
+    assert np.array_equal(f_colidx.cpu().numpy(), o_colidx)
+    assert np.array_equal(f_vals.cpu().numpy().astype(np.float64), o_vals)      # values are bit copies
+    # same structure as the full-output variant of the same kernels
+    (frp, fci, _), _, _ = run_and_compare(B, a, 1)
+    assert torch.equal(frp, f_rowptr) and torch.equal(fci, f_colidx)
+
+
+def test_mirror_rejects_upper_entries(B):
+    rp = torch.tensor([0, 1, 2], dtype=torch.int64, device="cuda")
+    ci = torch.tensor([1, 1], dtype=torch.int32, device="cuda")
+    cv = torch.tensor([1.0, 1.0], dtype=torch.float64, device="cuda")
+    with pytest.raises(B.SpsyrkError) as e:
+        B.spsyrk_mirror(2, rp, ci, cv)
+    assert e.value.status == 2
+
+
+# ---------------------------------------------------------------------------------- jaccard
+def test_jaccard(B):
+    a = W.small(2)
+    (rp, ci, cv), ref, plan = run_and_compare(B, a, 0)
+    rowptr_a = torch.from_numpy(a.rowptr).cuda()
+    jac = B.spsyrk_jaccard(a.m, 0, a.m, rowptr_a, rp, ci, cv).cpu().numpy()
+    exp = oracle.jaccard(0, a.m, a.rowptr, ref.rowptr, ref.colidx, oracle.to_int32(ref.vals))
+    assert np.all(np.abs(jac - exp) <= 1e-5 * np.abs(exp))
+    assert np.array_equal(jac, exp)                          # one correctly rounded division on both sides
+    rows = np.repeat(np.arange(a.m), np.diff(ref.rowptr))
+    assert np.all(jac[rows == ref.colidx] == 1.0)
+    # a row tile
+    r0, r1 = 1000, 1777
+    B.spsyrk_plan_set_rows(plan, r0, r1)
+    trp, tci, tcv, _ = B.tril_syrk(a.m, a.n, *dev(a), row_begin=r0, row_end=r1, plan=plan)
+    tj = B.spsyrk_jaccard(a.m, r0, r1 - r0, rowptr_a, trp, tci, tcv).cpu().numpy()
+    assert np.array_equal(tj, exp[ref.rowptr[r0]:ref.rowptr[r1]])
+
+
+# --------------------------------------------------------------------- host-buffer entry point
+def test_host_entry_point(B):
+    a = W.small(4)
+    rp, ci, cv = B.spsyrk_host_tril(a.m, a.n, torch.from_numpy(a.rowptr), torch.from_numpy(a.colidx),
+                                    torch.from_numpy(a.vals), pinned=False)
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL)
+    assert np.array_equal(rp.numpy(), ref.rowptr) and np.array_equal(ci.numpy(), ref.colidx)
+    check_values(cv.numpy(), ref, a.vals.dtype)
