@@ -185,7 +185,7 @@ class _DevArray:
     """A device pointer dressed as a CUDA array so that torch can wrap it without copying."""
 
     def __init__(self, ptr, count, typestr):
-        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (ptr, True), "version": 2}
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr, "data": (ptr, False), "version": 2}
 
 
 def spsyrk_mirror_workspace_bytes(m, nnz_l, dtype) -> int:
