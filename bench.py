@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the local sparse SYRK path: one JSON line per run.
+
+A step is one pass of the whole hot path over one matrix: plan (transpose, work estimate,
+binning), symbolic (count + scan), numeric, mirror, and the Jaccard normalisation when the
+matrix is int32.  The default workload is the large Erdos-Renyi configuration (the one the
+roofline target is quoted on).  `--impl reference` times the CPU oracle on a bounded sample
+of the same workload instead.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl ours|reference]
+
+Under torchrun (N > 1) every rank runs an independent replica of the step on its own GPU
+(the path does not shard: no collective on the data path); value = N * work / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_09713_b200 import workloads as W  # noqa: E402
+
+METRIC = "tril_syrk_useful_multiply_adds_per_s"
+UNIT = "MAC/s"
+# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
+# (bytes per useful multiply-add, multiplied by the launch's multiply-adds); None = not captured.
+NCU_TRAFFIC_BYTES_PER_MAC = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        rows = [s for t, s in self.samples if t0 - 0.05 <= t <= t1 + 0.15] or [s for _, s in self.samples]
+        mhz, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                mhz.append(float(f[0])); mx = float(f[1])
+            except Exception:
+                continue
+            for nm, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(mhz)}
+
+
+def class_of_rows(work, deg):
+    """The library's row classes, recomputed on the host for the roofline's byte counts."""
+    cls = np.full(work.shape, 7, dtype=np.int8)
+    cls[work <= 16384] = 6
+    light = (deg <= 32) & (work <= 512)
+    for c, hi in ((5, 512), (4, 256), (3, 128), (2, 64), (1, 32)):
+        cls[light & (work <= hi)] = c
+    cls[work == 0] = 0
+    return cls
+
+
+def algorithmic_bytes(deg, work, cnt, sv):
+    """Bytes the row-by-row method must move for a set of rows: per row of A 8 + d_i (4 + sv) read,
+    per multiply-add one (row id, value) entry of a column list read, per output nonzero one
+    (column id, value) written, per output row an 8-byte row pointer."""
+    return int((8 + deg * (4 + sv)).sum() + work.sum() * (4 + sv) + cnt.sum() * (4 + sv) + 8 * deg.size)
+
+
+def oracle_sample(a, steps, warmup):
+    """Times the CPU oracle on a contiguous block of rows from the middle of the matrix."""
+    import oracle
+    cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
+    # size the block for a few seconds of work: probe 1/512 of the rows first
+    r0 = a.m // 2
+    probe = max(1, a.m // 512)
+    t = time.perf_counter()
+    res = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, r0, min(a.m, r0 + probe), cols=cols)
+    dt = max(time.perf_counter() - t, 1e-6)
+    rate = max(float(res.work.sum()), 1.0) / dt
+    per_row = max(float(res.work.sum()) / probe, 1.0)
+    budget_s = 20.0 / max(steps + warmup, 1) if (steps + warmup) > 2 else 10.0
+    rows = int(min(a.m - r0, max(probe, rate * budget_s / per_row)))
+    times, macs, nnz = [], 0, 0
+    for it in range(warmup + steps):
+        t = time.perf_counter()
+        res = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, r0, r0 + rows, cols=cols)
+        dt = time.perf_counter() - t
+        if it >= warmup:
+            times.append(dt)
+        macs, nnz = int(res.work.sum()), res.nnz
+    return {"rows": rows, "r0": r0, "macs": macs, "nnz": nnz, "times": times}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    a = W.config(args.workload)
+    s = oracle_sample(a, args.steps, args.warmup)
+    ms = 1e3 * float(np.mean(s["times"]))
+    value = s["macs"] / (ms / 1e3)
+    sample = f"rows [{s['r0']}, {s['r0'] + s['rows']}) of {a.name}: {s['macs']} multiply-adds, {s['nnz']} output nonzeros per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64" if a.vals.dtype == np.float64 else ("f32" if a.vals.dtype == np.float32 else "i32"),
+            "data": "synthetic", "config": {"workload": a.name, "sample": sample},
+            "nnz_per_s": s["nnz"] / (ms / 1e3),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_09713_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    a = W.config(args.workload)
+    sv = a.vals.dtype.itemsize
+    dname = {np.dtype(np.float64): "f64", np.dtype(np.float32): "f32", np.dtype(np.int32): "i32"}[a.vals.dtype]
+    d_rowptr, d_colidx, d_vals = (torch.from_numpy(x).cuda() for x in (a.rowptr, a.colidx, a.vals))
+    is_int = a.vals.dtype == np.int32
+    do_mirror = not (args.no_mirror or args.workload == 2)  # the 1e5 x 1e5 dense mirror of config 2 is not asked for
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    mirror_ws = None
+
+    def step(timing=False, keep=False):
+        nonlocal mirror_ws
+        marks = [ev()]
+        plan = B.spsyrk_plan(a.m, a.n, d_rowptr, d_colidx, d_vals, mode=B.TRIL)
+        if timing:
+            B.spsyrk_plan_enable_timing(plan)
+        marks.append(ev())
+        c_rowptr = torch.empty(a.m + 1, dtype=torch.int64, device="cuda")
+        nnz = B.spsyrk_symbolic(plan, c_rowptr)
+        marks.append(ev())
+        c_colidx = torch.empty(max(nnz, 1), dtype=torch.int32, device="cuda")
+        c_vals = torch.empty(max(nnz, 1), dtype=d_vals.dtype, device="cuda")
+        B.spsyrk_numeric(plan, c_rowptr, c_colidx, c_vals)
+        marks.append(ev())
+        nnz_f = 0
+        if do_mirror:
+            if mirror_ws is None:
+                mirror_ws = torch.empty(B.spsyrk_mirror_workspace_bytes(a.m, nnz, d_vals.dtype), dtype=torch.uint8, device="cuda")
+            f = B.spsyrk_mirror(a.m, c_rowptr, c_colidx[:nnz], c_vals[:nnz], workspace=mirror_ws)
+            nnz_f = f[1].numel()
+            del f
+        marks.append(ev())
+        if is_int:
+            jac = B.spsyrk_jaccard(a.m, 0, a.m, d_rowptr, c_rowptr, c_colidx[:nnz], c_vals[:nnz])
+            del jac
+        marks.append(ev())
+        out = {"marks": marks, "nnz": nnz, "nnz_full": nnz_f, "plan": plan}
+        if keep:
+            out["c"] = (c_rowptr, c_colidx[:nnz], c_vals[:nnz])
+        return out
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 1)):
+        r = step()
+        torch.cuda.synchronize()
+        del r
+    launches0 = B.spsyrk_launch_count()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    t0 = time.time()
+    results = [step(timing=True) for _ in range(args.steps)]
+    barrier()
+    t1 = time.time()
+    launches = (B.spsyrk_launch_count() - launches0) // args.steps
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    total_ms = results[0]["marks"][0].elapsed_time(results[-1]["marks"][-1])
+    ms_per_step = total_ms / args.steps
+    if world > 1:
+        t = torch.tensor([ms_per_step], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step = float(t.item())
+    names = ["plan", "symbolic", "numeric", "mirror", "jaccard"]
+    phases = {nm: float(np.mean([r["marks"][i].elapsed_time(r["marks"][i + 1]) for r in results])) for i, nm in enumerate(names)}
+    work_total, class_rows = B.spsyrk_plan_stats(results[-1]["plan"])
+    nnz_c, nnz_f = results[-1]["nnz"], results[-1]["nnz_full"]
+    sym_ms = np.mean([B.spsyrk_plan_timings(r["plan"])[0] for r in results], axis=0)
+    num_ms = np.mean([B.spsyrk_plan_timings(r["plan"])[1] for r in results], axis=0)
+    value = world * work_total / (ms_per_step / 1e3)
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dname,
+            "data": "synthetic",
+            "config": {"workload": a.name, "m": a.m, "n": a.n, "nnz_a": a.nnz, "multiply_adds": work_total, "nnz_c_l": nnz_c,
+                       "nnz_full": nnz_f, "step": "plan+symbolic+numeric" + ("+mirror" if do_mirror else "") + ("+jaccard" if is_int else ""),
+                       "l2_policy": "inputs_larger_than_l2", "parallelism": f"replicas x{world}"},
+            "nnz_per_s": world * nnz_c / (ms_per_step / 1e3), "phases_ms": phases,
+            "numeric_class_ms": [float(x) for x in num_ms], "symbolic_class_ms": [float(x) for x in sym_ms],
+            "class_rows": class_rows, "gpu_launches": int(launches), "clocks": clocks}
+
+    if rank == 0 and not args.skip_extras:
+        # ---- roofline of the dominant kernel (the numeric launch of the heaviest row class)
+        peak, peak_kind = measured_peaks()
+        plan = results[-1]["plan"]
+        _, _, _, work_dev = B.spsyrk_plan_buffers(plan)
+        work = work_dev.cpu().numpy()
+        keep = step(keep=True)
+        torch.cuda.synchronize()
+        cnt = np.diff(keep["c"][0].cpu().numpy())
+        deg = np.diff(a.rowptr)
+        cls = class_of_rows(work, deg)
+        dom = int(np.argmax(num_ms))
+        sel = cls == dom
+        bytes_dom = algorithmic_bytes(deg[sel], work[sel], cnt[sel], sv)
+        ach = bytes_dom / (num_ms[dom] / 1e3) / 1e9
+        kernel = ("numeric_warp_kernel<N=%d>" % (16 << dom)) if dom <= 5 else ("rows_cta_kernel<%d threads, numeric>" % (256 if dom == 6 else 1024))
+        traffic = None
+        if NCU_TRAFFIC_BYTES_PER_MAC is not None:
+            traffic = NCU_TRAFFIC_BYTES_PER_MAC * float(work[sel].sum())
+        line["roofline"] = {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                            "traffic": traffic, "peak_kind": peak_kind, "algorithmic_bytes_per_launch": bytes_dom,
+                            "launch_ms": float(num_ms[dom]), "rows_in_launch": int(sel.sum()),
+                            "multiply_adds_in_launch": int(work[sel].sum())}
+        b_gust = algorithmic_bytes(deg, work, cnt, sv)
+        b_min = a.rowptr.nbytes + a.colidx.nbytes + a.vals.nbytes + 8 * (a.n + 1) + a.nnz * (4 + sv) + 8 * (a.m + 1) + nnz_c * (4 + sv)
+        line["numeric_pass"] = {"ms": phases["numeric"], "b_gust_bytes": b_gust, "b_min_bytes": int(b_min),
+                                "gbs_b_gust": b_gust / (phases["numeric"] / 1e3) / 1e9, "frac_of_peak": b_gust / (phases["numeric"] / 1e3) / 1e9 / peak,
+                                "frac_of_8tbs": b_gust / (phases["numeric"] / 1e3) / 1e9 / 8000.0}
+        if do_mirror:
+            mb = nnz_c * (4 + sv) + 8 * (a.m + 1) + nnz_f * (4 + sv) + 8 * (a.m + 1)
+            line["mirror_pass"] = {"ms": phases["mirror"], "bytes": int(mb), "gbs": mb / (phases["mirror"] / 1e3) / 1e9,
+                                   "frac_of_peak": mb / (phases["mirror"] / 1e3) / 1e9 / peak}
+        del keep
+        # ---- the full-output variant of the same kernels (symbolic + numeric only)
+        if not args.no_full:
+            fplan = B.spsyrk_plan(a.m, a.n, d_rowptr, d_colidx, d_vals, mode=B.FULL)
+            fw, _ = B.spsyrk_plan_stats(fplan)
+            tt = []
+            for it in range(3):
+                e0 = ev()
+                frp = torch.empty(a.m + 1, dtype=torch.int64, device="cuda")
+                fn = B.spsyrk_symbolic(fplan, frp)
+                e1 = ev()
+                fci = torch.empty(max(fn, 1), dtype=torch.int32, device="cuda")
+                fcv = torch.empty(max(fn, 1), dtype=d_vals.dtype, device="cuda")
+                B.spsyrk_numeric(fplan, frp, fci, fcv)
+                e2 = ev()
+                torch.cuda.synchronize()
+                tt.append((e0.elapsed_time(e1), e1.elapsed_time(e2)))
+                del frp, fci, fcv
+            fs, fnum = (float(np.mean([t[i] for t in tt[1:]])) for i in (0, 1))
+            line["full_variant"] = {"multiply_adds": fw, "nnz": fn, "symbolic_ms": fs, "numeric_ms": fnum,
+                                    "tril_speedup_numeric": fnum / phases["numeric"],
+                                    "tril_speedup_symbolic_plus_numeric": (fs + fnum) / (phases["symbolic"] + phases["numeric"])}
+            del fplan
+        torch.cuda.empty_cache()
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    if not args.skip_extras:
+        h_in = tuple(torch.from_numpy(x).pin_memory() for x in (a.rowptr, a.colidx, a.vals))
+        out = (torch.empty(a.m + 1, dtype=torch.int64, pin_memory=True), torch.empty(max(nnz_c, 1), dtype=torch.int32, pin_memory=True),
+               torch.empty(max(nnz_c, 1), dtype=d_vals.dtype, pin_memory=True))
+        del d_rowptr, d_colidx, d_vals, results, mirror_ws
+        torch.cuda.empty_cache()
+        B.spsyrk_host_tril(a.m, a.n, *h_in, out=out)  # warm-up
+        barrier()
+        ts = time.perf_counter()
+        for _ in range(args.steps):
+            B.spsyrk_host_tril(a.m, a.n, *h_in, out=out)
+        barrier()
+        e2e_ms = (time.perf_counter() - ts) * 1e3 / args.steps
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        h2d = a.rowptr.nbytes + a.colidx.nbytes + a.vals.nbytes
+        d2h = 8 * (a.m + 1) + nnz_c * (4 + sv)
+        line["e2e"] = {"value": world * work_total / (e2e_ms / 1e3), "unit": UNIT, "ms_per_step": e2e_ms,
+                       "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                       "what": "spsyrk_host_tril: H2D of A, plan+symbolic+numeric, D2H of C_L (mirror not included)"}
+
+    if rank == 0 and world == 1 and not args.skip_extras and not args.no_cpu:
+        s = oracle_sample(a, 1, 0)
+        line["cpu_baseline"] = {"value": s["macs"] / s["times"][0], "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"rows [{s['r0']}, {s['r0'] + s['rows']}) of {a.name}: {s['macs']} multiply-adds in {s['times'][0]:.2f} s"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=5, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--no-mirror", action="store_true")
+    ap.add_argument("--no-full", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--skip-extras", action="store_true", help="timed steps only (for profiler runs)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

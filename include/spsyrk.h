@@ -126,7 +126,8 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t *d_c_rowptr,
  * Three-step use:
  *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for (m, nnz_l, dtype).
  *   2. d_f_colidx == NULL: writes d_f_rowptr[m + 1] and *nnz_full_out (synchronises).
- *   3. all pointers set: fills d_f_colidx / d_f_vals using the d_f_rowptr of step 2.  Asynchronous.
+ *   3. all pointers set: fills d_f_colidx / d_f_vals using the d_f_rowptr of step 2 (synchronises once,
+ *      to size the per-class launches of its segment sort).
  * nnz_l = d_l_rowptr[m].  Errors: INVALID_ARG, WORKSPACE, BAD_CSR (an entry above the diagonal), CUDA.
  */
 spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
@@ -164,6 +165,19 @@ spsyrk_status_t spsyrk_plan_stats(spsyrk_plan_t plan, int64_t *work_total, int64
  */
 spsyrk_status_t spsyrk_plan_buffers(spsyrk_plan_t plan, const int64_t **d_colptr, const int32_t **d_at_row,
                                     const void **d_at_val, const int64_t **d_work);
+
+/*
+ * Measurement aids (no effect on results).
+ * spsyrk_plan_enable_timing : from now on spsyrk_symbolic / spsyrk_numeric record CUDA events on
+ *     the caller's stream around the launch of every row class.
+ * spsyrk_plan_timings       : device milliseconds of the last symbolic and numeric call per row
+ *     class (index = class, 0 unused); waits for those events.  A numeric entry is 0 if numeric
+ *     has not run since timing was enabled.
+ * spsyrk_launch_count       : kernels launched by this library in this process so far.
+ */
+spsyrk_status_t spsyrk_plan_enable_timing(spsyrk_plan_t plan);
+spsyrk_status_t spsyrk_plan_timings(spsyrk_plan_t plan, float symbolic_ms[8], float numeric_ms[8]);
+int64_t spsyrk_launch_count(void);
 
 void spsyrk_destroy(spsyrk_plan_t plan);
 

@@ -47,6 +47,12 @@ _lib.spsyrk_destroy.restype = None
 _lib.spsyrk_status_string.argtypes = [_int]
 _lib.spsyrk_status_string.restype = ctypes.c_char_p
 _lib.spsyrk_host_tril.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _vp, _vp, _int, _int, _vp, _i64p, _vp, _vp]
+_lib.spsyrk_plan_enable_timing.argtypes = [_vp]
+_lib.spsyrk_plan_timings.argtypes = [_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+_lib.spsyrk_launch_count.argtypes = []
+_lib.spsyrk_launch_count.restype = ctypes.c_int64
+for _name in ("spsyrk_plan_enable_timing", "spsyrk_plan_timings"):
+    getattr(_lib, _name).restype = _int
 for _name in ("spsyrk_plan", "spsyrk_plan_set_rows", "spsyrk_symbolic", "spsyrk_numeric", "spsyrk_mirror",
               "spsyrk_jaccard", "spsyrk_plan_stats", "spsyrk_plan_buffers", "spsyrk_host_tril"):
     getattr(_lib, _name).restype = _int
@@ -161,6 +167,22 @@ def spsyrk_plan_stats(plan: Plan):
     return work.value, list(cls)
 
 
+def spsyrk_plan_enable_timing(plan: Plan):
+    _check(_lib.spsyrk_plan_enable_timing(plan._h), "spsyrk_plan_enable_timing")
+
+
+def spsyrk_plan_timings(plan: Plan):
+    """(symbolic_ms[8], numeric_ms[8]): device milliseconds per row class of the last calls."""
+    sym = (ctypes.c_float * NCLASS)()
+    num = (ctypes.c_float * NCLASS)()
+    _check(_lib.spsyrk_plan_timings(plan._h, sym, num), "spsyrk_plan_timings")
+    return list(sym), list(num)
+
+
+def spsyrk_launch_count() -> int:
+    return int(_lib.spsyrk_launch_count())
+
+
 def spsyrk_plan_buffers(plan: Plan):
     """Copies of the plan's column lists and work estimate as torch tensors: (colptr, at_row, at_val, work)."""
     ptrs = [_vp() for _ in range(4)]
@@ -226,19 +248,24 @@ def spsyrk_jaccard(m, row_begin, rows, a_rowptr, c_rowptr, c_colidx, c_counts, o
     return out
 
 
-def spsyrk_host_tril(m, n, rowptr, colidx, vals, mode=TRIL, pinned=True):
+def spsyrk_host_tril(m, n, rowptr, colidx, vals, mode=TRIL, pinned=True, out=None):
     """Whole path on HOST tensors through the host-buffer entry point.  Returns host tensors
-    (c_rowptr, c_colidx, c_vals); the result buffers are pinned when `pinned`."""
+    (c_rowptr, c_colidx, c_vals); the result buffers are pinned when `pinned`, or taken from
+    `out` = (c_rowptr, c_colidx, c_vals) when given (they must be large enough)."""
     assert not rowptr.is_cuda and not colidx.is_cuda and not vals.is_cuda
     code = _DTYPE_CODE[vals.dtype]
     nnz = colidx.numel()
     sess = _vp()
-    c_rowptr = torch.empty(m + 1, dtype=torch.int64, pin_memory=pinned)
+    c_rowptr = out[0] if out is not None else torch.empty(m + 1, dtype=torch.int64, pin_memory=pinned)
     nnz_c = ctypes.c_int64(0)
     _check(_lib.spsyrk_host_tril(ctypes.byref(sess), m, n, nnz, _p(rowptr), _p(colidx), _p(vals), code, mode,
                                  _p(c_rowptr), ctypes.byref(nnz_c), None, None), "spsyrk_host_tril(symbolic)")
-    c_colidx = torch.empty(max(nnz_c.value, 1), dtype=torch.int32, pin_memory=pinned)
-    c_vals = torch.empty(max(nnz_c.value, 1), dtype=vals.dtype, pin_memory=pinned)
+    if out is not None:
+        c_colidx, c_vals = out[1], out[2]
+        assert c_colidx.numel() >= nnz_c.value and c_vals.numel() >= nnz_c.value
+    else:
+        c_colidx = torch.empty(max(nnz_c.value, 1), dtype=torch.int32, pin_memory=pinned)
+        c_vals = torch.empty(max(nnz_c.value, 1), dtype=vals.dtype, pin_memory=pinned)
     _check(_lib.spsyrk_host_tril(ctypes.byref(sess), m, n, nnz, None, None, None, code, mode, None, None,
                                  _p(c_colidx), _p(c_vals)), "spsyrk_host_tril(numeric)")
     return c_rowptr, c_colidx[:nnz_c.value], c_vals[:nnz_c.value]

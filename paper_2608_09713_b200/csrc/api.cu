@@ -7,7 +7,14 @@
 #include "rows_cta.cuh"
 #include "rows_warp.cuh"
 
+#include <atomic>
+
 using namespace spsyrk;
+
+namespace spsyrk {
+static std::atomic<long long> g_launches{0};
+void note_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace spsyrk
 
 namespace {
 
@@ -64,6 +71,10 @@ struct spsyrk_plan_s {
     int64_t work_total;
     bool have_symbolic;
     bool key64;
+    // optional per-class timing of the symbolic and numeric launches
+    bool timing;
+    cudaEvent_t ev_sym[NCLASS + 1];
+    cudaEvent_t ev_num[NCLASS + 1];
 };
 
 namespace {
@@ -115,6 +126,7 @@ void launch_fill(spsyrk_plan_s* pl, cudaStream_t st) {
     const int64_t threads = (int64_t)P.m * G;
     column_fill_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P.rowptr, P.colidx, P.m, P.n, P.colptr,
                                                                              pl->cursor, pl->keys, P.err);
+    note_launches(1);
 }
 
 template <int G>
@@ -122,6 +134,7 @@ void launch_row_work(spsyrk_plan_s* pl, cudaStream_t st) {
     const PlanDev& P = pl->dev;
     const int64_t threads = (int64_t)(P.r1 - P.r0) * G;
     row_work_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P, pl->cls, BLOCK_CLASS_MAX_WORK, pl->work_total_dev);
+    note_launches(1);
 }
 
 int group_width(int64_t nnz, int64_t m) {
@@ -134,6 +147,7 @@ void launch_colsort_group(spsyrk_plan_s* pl, int64_t first, int64_t count, cudaS
     if (count <= 0) return;
     const int64_t threads = count * G;
     column_sort_group_kernel<V, R, G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(pl->dev, pl->colperm + first, count, pl->keys);
+    note_launches(1);
 }
 
 template <typename V>
@@ -150,6 +164,7 @@ spsyrk_status_t sort_columns(spsyrk_plan_s* pl, const int64_t* cs, cudaStream_t 
         const size_t smem = (size_t)(cb >> 5) * 2 * sizeof(uint32_t);
         SPSYRK_CUDA_TRY(cudaFuncSetAttribute(column_sort_cta_kernel<V, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         column_sort_cta_kernel<V, 512><<<(unsigned)big, 512, smem, st>>>(pl->dev, pl->colperm + cs[7], pl->keys, cb);
+        note_launches(1);
     }
     SPSYRK_CUDA_TRY(cudaGetLastError());
     return SPSYRK_OK;
@@ -184,6 +199,7 @@ void launch_symbolic_warp(spsyrk_plan_s* pl, int c, cudaStream_t st) {
     if (count <= 0) return;
     symbolic_warp_kernel<N><<<(unsigned)((count + ROW_WARPS - 1) / ROW_WARPS), ROW_WARPS * 32, 0, st>>>(
         pl->dev, pl->perm + pl->class_start[c], count, pl->cnt);
+    note_launches(1);
 }
 
 template <typename V, int N, typename Key>
@@ -193,15 +209,26 @@ void launch_numeric_warp(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int3
     constexpr int NW = numeric_warps(N);
     numeric_warp_kernel<V, N, Key><<<(unsigned)((count + NW - 1) / NW), NW * 32, 0, st>>>(
         pl->dev, pl->perm + pl->class_start[c], count, c_rowptr, c_colidx, static_cast<V*>(c_vals));
+    note_launches(1);
+}
+
+inline void mark(spsyrk_plan_s* pl, cudaEvent_t* ev, int i, cudaStream_t st) {
+    if (pl->timing) cudaEventRecord(ev[i], st);
 }
 
 template <typename V, typename Key>
 void launch_numeric_warp_all(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    mark(pl, pl->ev_num, 1, st);
     launch_numeric_warp<V, 32, Key>(pl, 1, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 2, st);
     launch_numeric_warp<V, 64, Key>(pl, 2, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 3, st);
     launch_numeric_warp<V, 128, Key>(pl, 3, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 4, st);
     launch_numeric_warp<V, 256, Key>(pl, 4, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 5, st);
     launch_numeric_warp<V, 512, Key>(pl, 5, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 6, st);
 }
 
 uint32_t row_chunk_bits(const spsyrk_plan_s* pl, uint32_t cap) {
@@ -218,6 +245,7 @@ spsyrk_status_t launch_symbolic_cta(spsyrk_plan_s* pl, int c, cudaStream_t st) {
     auto kern = rows_cta_kernel<int32_t, THREADS, false>;
     SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, 0u, pl->cnt, nullptr, nullptr, nullptr);
+    note_launches(1);
     return SPSYRK_OK;
 }
 
@@ -239,6 +267,7 @@ spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_
     SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, c_rowptr, c_colidx,
                                                   static_cast<V*>(c_vals));
+    note_launches(1);
     return SPSYRK_OK;
 }
 
@@ -248,8 +277,10 @@ spsyrk_status_t numeric_typed(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_
     else launch_numeric_warp_all<V, uint32_t>(pl, c_rowptr, c_colidx, c_vals, st);
     spsyrk_status_t s = launch_numeric_cta<V, 256>(pl, 6, BLOCK_ACC_SLOTS, c_rowptr, c_colidx, c_vals, st);
     if (s != SPSYRK_OK) return s;
+    mark(pl, pl->ev_num, 7, st);
     s = launch_numeric_cta<V, 1024>(pl, 7, 0u, c_rowptr, c_colidx, c_vals, st);
     if (s != SPSYRK_OK) return s;
+    mark(pl, pl->ev_num, 8, st);
     SPSYRK_CUDA_TRY(cudaGetLastError());
     return SPSYRK_OK;
 }
@@ -298,6 +329,7 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     }
     // 1. row pointers must be sane before anything indexes with them
     validate_rowptr_kernel<<<(unsigned)((m + 1 + 255) / 256), 256, 0, st>>>(d_rowptr, m, nnz, P.err);
+    note_launches(1);
     PLAN_TRY(cudaGetLastError());
     spsyrk_status_t s = read_err(pl, st);
     if (s != SPSYRK_OK) return fail(s);
@@ -305,6 +337,7 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     if (nnz > 0) {
         const unsigned hb = (unsigned)std::min<int64_t>((nnz + 255) / 256, 148 * 32);
         column_histogram_kernel<<<hb, 256, 0, st>>>(d_colidx, nnz, P.n, pl->colcnt, P.err);
+        note_launches(1);
     }
     PLAN_TRY(exclusive_scan_i64<uint32_t>(pl->colcnt, n, P.colptr, pl->partials, st));
     if (nnz > 0) {
@@ -315,7 +348,10 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
             default: launch_fill<32>(pl, st); break;
         }
     }
-    if (n > 0) column_class_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(P.colptr, P.n, pl->cls);
+    if (n > 0) {
+        column_class_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(P.colptr, P.n, pl->cls);
+        note_launches(1);
+    }
     PLAN_TRY(bin_items(pl->cls, n, pl->colperm, pl->class_start_dev, pl->blockhist, pl->offsets, pl->partials, st));
     int64_t cs[NCLASS + 1];
     PLAN_TRY(cudaMemcpyAsync(cs, pl->class_start_dev, sizeof(cs), cudaMemcpyDeviceToHost, st));
@@ -344,15 +380,23 @@ spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t* d_c_rowptr, int64_t
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int64_t rows = pl->dev.r1 - pl->dev.r0;
     if (rows > 0) SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->cnt, 0, (size_t)rows * sizeof(int32_t), st));
+    mark(pl, pl->ev_sym, 1, st);
     launch_symbolic_warp<32>(pl, 1, st);
+    mark(pl, pl->ev_sym, 2, st);
     launch_symbolic_warp<64>(pl, 2, st);
+    mark(pl, pl->ev_sym, 3, st);
     launch_symbolic_warp<128>(pl, 3, st);
+    mark(pl, pl->ev_sym, 4, st);
     launch_symbolic_warp<256>(pl, 4, st);
+    mark(pl, pl->ev_sym, 5, st);
     launch_symbolic_warp<512>(pl, 5, st);
+    mark(pl, pl->ev_sym, 6, st);
     spsyrk_status_t s = launch_symbolic_cta<256>(pl, 6, st);
     if (s != SPSYRK_OK) return s;
+    mark(pl, pl->ev_sym, 7, st);
     s = launch_symbolic_cta<1024>(pl, 7, st);
     if (s != SPSYRK_OK) return s;
+    mark(pl, pl->ev_sym, 8, st);
     SPSYRK_CUDA_TRY(cudaGetLastError());
     SPSYRK_CUDA_TRY(exclusive_scan_i64<int32_t>(pl->cnt, rows, d_c_rowptr, pl->partials, st));
     int64_t nnz = 0;
@@ -396,7 +440,40 @@ spsyrk_status_t spsyrk_plan_buffers(spsyrk_plan_t plan, const int64_t** d_colptr
     return SPSYRK_OK;
 }
 
-void spsyrk_destroy(spsyrk_plan_t plan) { delete plan; }
+void spsyrk_destroy(spsyrk_plan_t plan) {
+    if (!plan) return;
+    if (plan->timing)
+        for (int i = 0; i <= NCLASS; ++i) { cudaEventDestroy(plan->ev_sym[i]); cudaEventDestroy(plan->ev_num[i]); }
+    delete plan;
+}
+
+spsyrk_status_t spsyrk_plan_enable_timing(spsyrk_plan_t plan) {
+    if (!plan) return SPSYRK_ERR_INVALID_ARG;
+    if (plan->timing) return SPSYRK_OK;
+    for (int i = 0; i <= NCLASS; ++i) {
+        SPSYRK_CUDA_TRY(cudaEventCreate(&plan->ev_sym[i]));
+        SPSYRK_CUDA_TRY(cudaEventCreate(&plan->ev_num[i]));
+    }
+    plan->timing = true;
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_plan_timings(spsyrk_plan_t plan, float symbolic_ms[8], float numeric_ms[8]) {
+    if (!plan || !plan->timing || !symbolic_ms || !numeric_ms) return SPSYRK_ERR_INVALID_ARG;
+    if (!plan->have_symbolic) return SPSYRK_ERR_SEQUENCE;
+    symbolic_ms[0] = numeric_ms[0] = 0.f;
+    for (int c = 1; c < NCLASS; ++c) {
+        symbolic_ms[c] = numeric_ms[c] = 0.f;
+        SPSYRK_CUDA_TRY(cudaEventSynchronize(plan->ev_sym[c + 1]));
+        SPSYRK_CUDA_TRY(cudaEventElapsedTime(&symbolic_ms[c], plan->ev_sym[c], plan->ev_sym[c + 1]));
+        if (cudaEventQuery(plan->ev_num[c + 1]) == cudaSuccess && cudaEventQuery(plan->ev_num[c]) == cudaSuccess)
+            cudaEventElapsedTime(&numeric_ms[c], plan->ev_num[c], plan->ev_num[c + 1]);
+    }
+    cudaGetLastError();
+    return SPSYRK_OK;
+}
+
+int64_t spsyrk_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 const char* spsyrk_status_string(spsyrk_status_t s) {
     switch (s) {

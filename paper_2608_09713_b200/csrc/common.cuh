@@ -22,6 +22,9 @@ enum : uint32_t {
 
 constexpr int NCLASS = 8;  // row / column classes produced by the binning pass
 
+// kernel-launch bookkeeping behind spsyrk_launch_count (defined in api.cu)
+void note_launches(int n);
+
 #define SPSYRK_CUDA_TRY(expr)                                  \
     do {                                                       \
         cudaError_t _e = (expr);                               \
@@ -202,6 +205,7 @@ inline cudaError_t exclusive_scan_i64(const InT* in, int64_t n, int64_t* out, in
     scan_tile_sums_kernel<InT><<<(unsigned)ntiles, SCAN_THREADS, 0, st>>>(in, n, partials);
     scan_partials_kernel<<<1, 1024, 0, st>>>(partials, ntiles);
     scan_tiles_kernel<InT><<<(unsigned)ntiles, SCAN_THREADS, 0, st>>>(in, n, partials, out);
+    note_launches(3);
     return cudaGetLastError();
 }
 
@@ -282,6 +286,7 @@ inline cudaError_t bin_items(const uint8_t* cls, int64_t n, int32_t* perm, int64
     if (e != cudaSuccess) return e;
     bin_scatter_kernel<<<(unsigned)nb, BIN_THREADS, 0, st>>>(cls, n, offsets, nb, perm);
     bin_class_starts_kernel<<<1, 32, 0, st>>>(offsets, nb, class_start);
+    note_launches(3);
     return cudaGetLastError();
 }
 

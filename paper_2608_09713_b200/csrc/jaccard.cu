@@ -63,6 +63,7 @@ extern "C" spsyrk_status_t spsyrk_jaccard(int64_t m, int64_t row_begin, int64_t 
     if (blocks >= (int64_t(1) << 31)) return SPSYRK_ERR_OVERFLOW;
     jaccard_kernel<<<(unsigned)blocks, JAC_THREADS, 0, st>>>(row_begin, rows, nnz, d_a_rowptr, d_c_rowptr, d_c_colidx,
                                                              d_c_counts, d_jaccard);
+    note_launches(1);
     SPSYRK_CUDA_TRY(cudaGetLastError());
     return SPSYRK_OK;
 }

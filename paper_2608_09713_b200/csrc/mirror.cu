@@ -207,6 +207,7 @@ void launch_sort_warp(const MirrorWs& w, const int64_t* cs, int c, const int64_t
     if (count <= 0) return;
     mirror_sort_warp_kernel<V, R, Key><<<(unsigned)((count * 32 + 255) / 256), 256, 0, st>>>(
         w.perm + cs[c], count, l_rowptr, f_rowptr, w.stage_row, static_cast<const V*>(w.stage_val), f_colidx, static_cast<V*>(f_vals));
+    note_launches(1);
 }
 
 template <typename V, typename Key>
@@ -237,6 +238,7 @@ spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const i
     }
 #undef SCATTER
     mirror_class_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(l_rowptr, f_rowptr, m, w.cls);
+    note_launches(2);  // scatter + class
     SPSYRK_CUDA_TRY(bin_items(w.cls, m, w.perm, w.class_start_dev, w.blockhist, w.offsets, w.partials, st));
     int64_t cs[NCLASS + 1];
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(cs, w.class_start_dev, sizeof(cs), cudaMemcpyDeviceToHost, st));
@@ -251,6 +253,7 @@ spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const i
         auto kern = mirror_sort_cta_kernel<V, 512>;
         SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         kern<<<(unsigned)big, 512, smem, st>>>(w.perm + cs[7], m, cb, l_rowptr, f_rowptr, w.stage_row, sv, f_colidx, fv);
+        note_launches(1);
     }
     SPSYRK_CUDA_TRY(cudaGetLastError());
     return SPSYRK_OK;
@@ -292,6 +295,7 @@ extern "C" spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_
             }
 #undef COUNT
             mirror_rowtot_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(d_l_rowptr, w.ucnt, m, w.rowtot);
+            note_launches(2);  // count + row totals
         }
         SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(w.rowtot, m, d_f_rowptr, w.partials, st));
         int64_t nnz = 0;
