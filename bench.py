@@ -164,6 +164,8 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     a = W.config(args.workload)
+    if args.er_log2m:
+        a = W.erdos_renyi(1 << args.er_log2m, 1 << args.er_log2m, 16, W.SEED + 5, np.float64, -1.0, 1.0)
     sv = a.vals.dtype.itemsize
     dname = {np.dtype(np.float64): "f64", np.dtype(np.float32): "f32", np.dtype(np.int32): "i32"}[a.vals.dtype]
     d_rowptr, d_colidx, d_vals = (torch.from_numpy(x).cuda() for x in (a.rowptr, a.colidx, a.vals))
@@ -356,6 +358,8 @@ def main():
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--skip-extras", action="store_true", help="timed steps only (for profiler runs)")
+    ap.add_argument("--er-log2m", type=int, default=0,
+                    help="profiling aid: replace the workload by the large Erdos-Renyi recipe at m = n = 2**k")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -81,13 +81,41 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T* scratch, T* total) {
 // lane, ascending.  Element e of a group lives in lane (e / R) of the group, register e % R, so
 // that compare-exchanges at a distance below R stay inside a lane and the others are one
 // shuffle per register.  After the call lane l of a group holds sorted elements [l*R, l*R+R).
+//
+// Every compare-exchange is a plain min/max: merge levels whose direction depends on the
+// register index are resolved at compile time, and levels whose direction depends on the lane
+// run on complemented keys in the descending lanes (x -> ~x reverses the order), so that the
+// whole level is an ascending merge.
 // ---------------------------------------------------------------------------------------
+template <typename K>
+__device__ __forceinline__ K kmin(K a, K b) { return a < b ? a : b; }
+template <typename K>
+__device__ __forceinline__ K kmax(K a, K b) { return a < b ? b : a; }
+template <>
+__device__ __forceinline__ uint32_t kmin<uint32_t>(uint32_t a, uint32_t b) { return min(a, b); }
+template <>
+__device__ __forceinline__ uint32_t kmax<uint32_t>(uint32_t a, uint32_t b) { return max(a, b); }
+
 template <typename K, int R, int G = 32>
 __device__ __forceinline__ void group_bitonic_sort(K (&x)[R]) {
     static_assert((R & (R - 1)) == 0 && (G & (G - 1)) == 0 && G <= 32, "powers of two");
     const int gl = lane_id() & (G - 1);
+    bool flipped = false;
 #pragma unroll
     for (int k = 2; k <= G * R; k <<= 1) {
+        if (k >= R && k < G * R) {
+            // direction of this level is per lane: descending lanes work on complemented keys
+            const bool want = (gl & (k / R)) != 0;
+            const K m = (want != flipped) ? ~K(0) : K(0);
+#pragma unroll
+            for (int r = 0; r < R; ++r) x[r] ^= m;
+            flipped = want;
+        } else if (k == G * R && G * R > R) {
+            const K m = flipped ? ~K(0) : K(0);
+#pragma unroll
+            for (int r = 0; r < R; ++r) x[r] ^= m;
+            flipped = false;
+        }
 #pragma unroll
         for (int j = k >> 1; j > 0; j >>= 1) {
             if (j < R) {
@@ -95,11 +123,11 @@ __device__ __forceinline__ void group_bitonic_sort(K (&x)[R]) {
                 for (int r = 0; r < R; ++r) {
                     const int pr = r ^ j;
                     if (pr > r) {
-                        const bool up = (((gl * R + r) & k) == 0);
-                        K a = x[r], b = x[pr];
-                        const bool sw = (a > b) == up;
-                        x[r] = sw ? b : a;
-                        x[pr] = sw ? a : b;
+                        // for k < R the direction depends on r only (compile time); otherwise ascending
+                        const bool up = (k < R) ? ((r & k) == 0) : true;
+                        const K lo = kmin(x[r], x[pr]), hi = kmax(x[r], x[pr]);
+                        x[r] = up ? lo : hi;
+                        x[pr] = up ? hi : lo;
                     }
                 }
             } else {
@@ -107,12 +135,8 @@ __device__ __forceinline__ void group_bitonic_sort(K (&x)[R]) {
                 const bool lower = (gl & lj) == 0;
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    K other = __shfl_xor_sync(FULL_MASK, x[r], lj);
-                    const bool up = (((gl * R + r) & k) == 0);
-                    const bool keepmin = (lower == up);
-                    K mn = x[r] < other ? x[r] : other;
-                    K mx = x[r] < other ? other : x[r];
-                    x[r] = keepmin ? mn : mx;
+                    const K other = __shfl_xor_sync(FULL_MASK, x[r], lj);
+                    x[r] = lower ? kmin(x[r], other) : kmax(x[r], other);
                 }
             }
         }
