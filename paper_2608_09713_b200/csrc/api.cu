@@ -55,6 +55,7 @@ struct spsyrk_plan_s {
     int64_t rows_cap;
     // workspace views
     int32_t* perm;
+    uint4* hdr;  // per-row headers in class order
     int32_t* cnt;
     uint8_t* cls;
     uint64_t* keys;
@@ -71,6 +72,7 @@ struct spsyrk_plan_s {
     int64_t work_total;
     bool have_symbolic;
     bool key64;
+    int sm_count;
     // optional per-class timing of the symbolic and numeric launches
     bool timing;
     cudaEvent_t ev_sym[NCLASS + 1];
@@ -89,6 +91,7 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     auto desc = c.take<uint2>(nnz);
     auto work = c.take<int64_t>(m);
     auto perm = c.take<int32_t>(m);
+    auto hdr = c.take<uint4>(m);
     auto cnt = c.take<int32_t>(m);
     auto cls = c.take<uint8_t>(items);
     auto keys = c.take<uint64_t>(nnz);
@@ -104,7 +107,7 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     if (pl) {
         pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.desc = desc;
         pl->dev.work = work; pl->dev.err = err;
-        pl->perm = perm; pl->cnt = cnt; pl->cls = cls; pl->keys = keys; pl->colcnt = colcnt; pl->cursor = cursor;
+        pl->perm = perm; pl->hdr = hdr; pl->cnt = cnt; pl->cls = cls; pl->keys = keys; pl->colcnt = colcnt; pl->cursor = cursor;
         pl->colperm = colperm; pl->blockhist = blockhist; pl->offsets = offsets; pl->partials = partials;
         pl->class_start_dev = class_start_dev; pl->work_total_dev = work_total_dev;
     }
@@ -185,6 +188,10 @@ spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
         }
     }
     SPSYRK_CUDA_TRY(bin_items(pl->cls, rows, pl->perm, pl->class_start_dev, pl->blockhist, pl->offsets, pl->partials, st));
+    if (rows > 0) {
+        row_header_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(P, pl->perm, rows, pl->hdr);
+        note_launches(1);
+    }
     unsigned long long wt = 0;
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(pl->class_start, pl->class_start_dev, sizeof(pl->class_start), cudaMemcpyDeviceToHost, st));
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(&wt, pl->work_total_dev, sizeof(wt), cudaMemcpyDeviceToHost, st));
@@ -207,8 +214,15 @@ void launch_numeric_warp(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int3
     const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
     if (count <= 0) return;
     constexpr int NW = numeric_warps(N);
-    numeric_warp_kernel<V, N, Key><<<(unsigned)((count + NW - 1) / NW), NW * 32, 0, st>>>(
-        pl->dev, pl->perm + pl->class_start[c], count, c_rowptr, c_colidx, static_cast<V*>(c_vals));
+    // persistent warps: exactly as many CTAs as are resident at once, each warp walks its rows with
+    // a stride of the whole grid
+    auto kern = numeric_warp_kernel<V, N, Key>;
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const int64_t want = (count + NW - 1) / NW;
+    const int64_t cap = (int64_t)pl->sm_count * per_sm;
+    kern<<<(unsigned)std::min(want, cap), NW * 32, 0, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, c_rowptr, c_colidx,
+                                                            static_cast<V*>(c_vals));
     note_launches(1);
 }
 
@@ -318,6 +332,11 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     pl->dtype = dtype;
     pl->rows_cap = m;
     pl->key64 = m > (int64_t(1) << 22);
+    {
+        int dev_id = 0;
+        pl->sm_count = 148;
+        if (cudaGetDevice(&dev_id) == cudaSuccess) cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, dev_id);
+    }
     carve(pl, d_workspace, m, n, nnz, sv);
 
     auto fail = [&](spsyrk_status_t s) { delete pl; return s; };

@@ -16,7 +16,9 @@ namespace spsyrk {
 
 constexpr int ROW_WARPS = 8;  // warps (rows) per CTA in the symbolic warp-class kernel
 // warps per CTA of the numeric warp-class kernel: keeps static shared memory under 48 KB
-__host__ __device__ constexpr int numeric_warps(int n) { return n >= 512 ? 4 : 8; }
+__host__ __device__ constexpr int numeric_warps(int n) { return n >= 512 ? 2 : n >= 256 ? 4 : 8; }
+// register budget: at least this many CTAs of the numeric kernel must fit on an SM
+__host__ __device__ constexpr int numeric_min_ctas(int n) { return n == 256 ? 6 : 1; }
 
 template <int N>
 __global__ void __launch_bounds__(ROW_WARPS * 32) symbolic_warp_kernel(PlanDev P, const int32_t* __restrict__ rows, int64_t nrows,
@@ -66,8 +68,35 @@ __global__ void __launch_bounds__(ROW_WARPS * 32) symbolic_warp_kernel(PlanDev P
     if (lane == 0) cnt[rloc] = local;
 }
 
+// Asynchronous global -> shared copies of 4 or 8 bytes (no register staging), grouped per thread.
+template <int BYTES>
+__device__ __forceinline__ void cp_async(void* smem_dst, const void* gmem_src) {
+    static_assert(BYTES == 4 || BYTES == 8, "cp.async size");
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2;\n" ::"r"(dst), "l"(gmem_src), "n"(BYTES) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int KEEP>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(KEEP) : "memory"); }
+
+// Per-row header in class order, written by the plan: the row's index inside the plan's range, the
+// position of its first nonzero in A and its number of nonzeros.
+__global__ void __launch_bounds__(256) row_header_kernel(PlanDev P, const int32_t* __restrict__ perm, int64_t rows,
+                                                         uint4* __restrict__ hdr) {
+    const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= rows) return;
+    const int32_t rloc = perm[n];
+    const int64_t i = (int64_t)P.r0 + rloc;
+    const int64_t p0 = P.rowptr[i], p1 = P.rowptr[i + 1];
+    hdr[n] = make_uint4((uint32_t)rloc, (uint32_t)p0, (uint32_t)(p1 - p0), 0u);
+}
+
+// Numeric pass for light rows, one warp per row, software-pipelined over the rows a warp owns:
+// while row n is sorted and written, the column-list entries of row n+1 stream into shared memory
+// through cp.async, the descriptors of row n+2 and the header of row n+3 are in flight in
+// registers.  Memory latency is hidden inside the warp instead of by occupancy.
 template <typename V, int N, typename Key>
-__global__ void __launch_bounds__(numeric_warps(N) * 32) numeric_warp_kernel(PlanDev P, const int32_t* __restrict__ rows, int64_t nrows,
+__global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows,
                                                                       const int64_t* __restrict__ c_rowptr,
                                                                       int32_t* __restrict__ c_colidx, V* __restrict__ c_vals) {
     using Acc = typename AccOf<V>::type;
@@ -75,108 +104,161 @@ __global__ void __launch_bounds__(numeric_warps(N) * 32) numeric_warp_kernel(Pla
     constexpr int R = N / 32;
     constexpr int IDXB = ilog2_ce(N);
     constexpr Key PAD = ~Key(0);
-    __shared__ Acc s_val[NW][N];      // products by item index t; later the compacted output values
-    __shared__ int32_t s_oj[NW][N];   // compacted output column ids
-    __shared__ Acc s_a[NW][32];       // a_ik per list
-    __shared__ uint32_t s_smo[NW][32];  // list start minus list offset: item t of list s is entry t + smo[s]
+    // double-buffered landing zones of the gathers; buffer b is reused for row n's products and
+    // then for its compacted output
+    // the output staging indexes these arrays through pad(): one spare slot per eight keeps the
+    // stride-R writes of the compaction off a single bank
+    constexpr int NP = N + N / 8;
+    __shared__ uint32_t s_j[NW][2][NP];
+    __shared__ Acc s_v[NW][2][NP];
+    __shared__ uint8_t s_own[NW][2][N];
+    __shared__ Acc s_a[NW][2][32];
     const int warp = threadIdx.x >> 5, lane = lane_id();
-    const int64_t widx = (int64_t)blockIdx.x * NW + warp;
-    if (widx >= nrows) return;
-    const int32_t rloc = rows[widx];
-    const int64_t i = (int64_t)P.r0 + rloc;
-    const int64_t p0 = P.rowptr[i];
-    const int deg = (int)(P.rowptr[i + 1] - p0);
-    const bool live = lane < deg;
-    uint2 d = live ? P.desc[p0 + lane] : make_uint2(0u, 0u);
-    const uint32_t incl = warp_inclusive_scan(d.y);
-    const uint32_t w = __shfl_sync(FULL_MASK, incl, 31);
-    const uint32_t off = live ? incl - d.y : 0xffffffffu;  // first item of this lane's list
-    s_smo[warp][lane] = d.x - off;
-    s_a[warp][lane] = live ? (Acc) static_cast<const V*>(P.vals)[p0 + lane] : Acc(0);
-    __syncwarp();
+    const int64_t stride = (int64_t)gridDim.x * NW;
+    int64_t n = (int64_t)blockIdx.x * NW + warp;
+    if (n >= nrows) return;
 
-    Key key[R];
+    const uint4 none = make_uint4(0u, 0u, 0u, 0u);
+    auto load_hdr = [&](int64_t idx) { return idx < nrows ? hdr[idx] : none; };
+    auto load_desc = [&](const uint4& h) { return (uint32_t)lane < h.z ? P.desc[(int64_t)h.y + lane] : make_uint2(0u, 0u); };
+    auto load_a = [&](const uint4& h) { return (uint32_t)lane < h.z ? (Acc) static_cast<const V*>(P.vals)[(int64_t)h.y + lane] : Acc(0); };
+    // issue the gathers of one row into buffer b; returns its item count
+    auto issue = [&](const uint4& h, const uint2& d, Acc a, int b) -> uint32_t {
+        const bool live = (uint32_t)lane < h.z;
+        const uint32_t incl = warp_inclusive_scan(d.y);
+        const uint32_t w = __shfl_sync(FULL_MASK, incl, 31);
+        const uint32_t off = live ? incl - d.y : 0xffffffffu;  // first item of this lane's list
+        const uint32_t smo = d.x - off;                        // item t of this list is entry t + smo
+        s_a[warp][b][lane] = a;
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        key[r] = PAD;
-        if ((uint32_t)(r * 32) < w) {  // warp-uniform
-            // owner list of item t = 32 r + lane: the list active at item 32 r, plus the lists that
-            // start inside (32 r, t]; starts are distinct because every list has at least one item
-            const uint32_t rel = off - (uint32_t)(r * 32);  // in 1..31 iff the list starts inside this round
-            const uint32_t before = __popc(__ballot_sync(FULL_MASK, off <= (uint32_t)(r * 32)));
-            const uint32_t startbits = __reduce_or_sync(FULL_MASK, (rel - 1u < 31u) ? (1u << rel) : 0u);
-            const uint32_t s = before - 1u + __popc(startbits & (0xfffffffeu >> (31 - lane)));
+        for (int r = 0; r < R; ++r) {
+            if ((uint32_t)(r * 32) < w) {  // warp-uniform
+                // owner list of item t = 32 r + lane: the list active at item 32 r plus the lists that
+                // start inside (32 r, t]; starts are distinct because every list has at least one item
+                const uint32_t rel = off - (uint32_t)(r * 32);
+                const uint32_t before = __popc(__ballot_sync(FULL_MASK, off <= (uint32_t)(r * 32)));
+                const uint32_t startbits = __reduce_or_sync(FULL_MASK, (rel - 1u < 31u) ? (1u << rel) : 0u);
+                const uint32_t s = before - 1u + __popc(startbits & (0xfffffffeu >> (31 - lane)));
+                const uint32_t q = r * 32 + lane + __shfl_sync(FULL_MASK, smo, s & 31);
+                const uint32_t t = r * 32 + lane;
+                if (t < w) {
+                    cp_async<4>(&s_j[warp][b][t], P.at_row + q);
+                    cp_async<sizeof(V)>(&s_v[warp][b][t], static_cast<const V*>(P.at_val) + q);
+                    s_own[warp][b][t] = (uint8_t)s;
+                }
+            }
+        }
+        cp_async_commit();
+        return w;
+    };
+
+    // prologue
+    uint4 h0 = load_hdr(n), hB = load_hdr(n + stride), hA = load_hdr(n + 2 * stride);
+    uint2 d0 = load_desc(h0);
+    Acc a0 = load_a(h0);
+    uint2 dB = load_desc(hB);
+    Acc aB = load_a(hB);
+    uint32_t rloc_n = h0.x;
+    int64_t ob_n = c_rowptr[rloc_n];
+    uint32_t w_n = issue(h0, d0, a0, 0);
+    int b = 0;
+
+    for (; n < nrows; n += stride, b ^= 1) {
+        // stage A: header of row n+3; stage B: descriptors of row n+2; stage C: gathers of row n+1
+        const uint4 hNew = load_hdr(n + 3 * stride);
+        const uint2 dNew = load_desc(hA);
+        const Acc aNew = load_a(hA);
+        const int64_t ob_next = hB.z ? c_rowptr[hB.x] : 0;
+        const uint32_t w_next = issue(hB, dB, aB, b ^ 1);
+
+        // stage D: row n.  Its gathers were committed one group ago.
+        cp_async_wait<1>();
+        __syncwarp();
+        Key key[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            key[r] = PAD;
             const uint32_t t = r * 32 + lane;
-            if (t < w) {
-                const uint32_t q = t + s_smo[warp][s];
-                const uint32_t j = (uint32_t)P.at_row[q];
-                const Acc v = (Acc) static_cast<const V*>(P.at_val)[q];
-                s_val[warp][t] = acc_mul(s_a[warp][s], v);
+            if (t < w_n) {
+                const uint32_t j = s_j[warp][b][t];
+                const Acc v = (Acc) * reinterpret_cast<const V*>(&s_v[warp][b][t]);
+                s_v[warp][b][t] = acc_mul(s_a[warp][b][s_own[warp][b][t]], v);
                 key[r] = ((Key)j << IDXB) | (Key)t;
             }
         }
-    }
-    group_bitonic_sort<Key, R, 32>(key);
-    __syncwarp();
+        group_bitonic_sort<Key, R, 32>(key);
+        __syncwarp();
 
-    // products in sorted order with an ordered segmented sum inside the lane: after it the last
-    // element of a run of equal j holds the run's sum as far as this lane can see
-    Acc sum[R];
+        // same[r]: element r continues the run of equal j of element r-1 (same[0]: of the previous
+        // lane's last element).  Padding keys sort to the end and never equal a real j.
+        constexpr Key JUNIT = Key(1) << IDXB;
+        const Key prev_last = __shfl_up_sync(FULL_MASK, key[R - 1], 1);
+        bool same[R + 1];
+        same[0] = lane > 0 && ((key[0] ^ prev_last) < JUNIT);
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const Acc v = key[r] != PAD ? s_val[warp][(uint32_t)(key[r] & (Key)(N - 1))] : Acc(0);
-        sum[r] = (r > 0 && (key[r] >> IDXB) == (key[r > 0 ? r - 1 : 0] >> IDXB)) ? acc_add(sum[r > 0 ? r - 1 : 0], v) : v;
-    }
-    // runs that continue from the previous lane: restart the leading run from the carried sum, in
-    // order; repeat while a lane that is one single run passes a changed sum on (almost never)
-    const Key firstj = key[0] >> IDXB;
-    const Key prevj = __shfl_up_sync(FULL_MASK, key[R - 1] >> IDXB, 1);
-    const bool joins = lane > 0 && key[0] != PAD && prevj == firstj;
-    for (int iter = 0; iter < 32; ++iter) {
-        const Acc carry = __shfl_up_sync(FULL_MASK, sum[R - 1], 1);
-        const Acc old_tail = sum[R - 1];
-        if (joins) {
-            Acc acc = carry;
-            bool in_run = true;
+        for (int r = 1; r < R; ++r) same[r] = (key[r] ^ key[r - 1]) < JUNIT;
+        same[R] = __shfl_down_sync(FULL_MASK, same[0] ? 1 : 0, 1) != 0 && lane < 31;
+        // products in sorted order with an ordered segmented sum inside the lane: after it the last
+        // element of a run holds the run's sum as far as this lane can see
+        Acc sum[R];
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                in_run = in_run && ((key[r] >> IDXB) == firstj) && key[r] != PAD;
-                if (in_run) { acc = acc_add(acc, s_val[warp][(uint32_t)(key[r] & (Key)(N - 1))]); sum[r] = acc; }
+        for (int r = 0; r < R; ++r) {
+            const Acc v = s_v[warp][b][(uint32_t)(key[r] & (Key)(N - 1))];
+            sum[r] = (r > 0 && same[r]) ? acc_add(sum[r > 0 ? r - 1 : 0], v) : v;
+        }
+        // runs that continue from the previous lane: restart the leading run from the carried sum, in
+        // order; repeat while a lane that is one single run passes a changed sum on (almost never)
+        const bool joins = same[0] && key[0] != PAD;
+        if (__any_sync(FULL_MASK, joins)) {
+            for (int iter = 0; iter < 32; ++iter) {
+                const Acc carry = __shfl_up_sync(FULL_MASK, sum[R - 1], 1);
+                const Acc old_tail = sum[R - 1];
+                if (joins) {
+                    Acc acc = carry;
+                    bool in_run = true;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        in_run = in_run && (r == 0 || same[r]);
+                        if (in_run) { acc = acc_add(acc, s_v[warp][b][(uint32_t)(key[r] & (Key)(N - 1))]); sum[r] = acc; }
+                    }
+                }
+                if (!__any_sync(FULL_MASK, joins && !(sum[R - 1] == old_tail))) break;
             }
         }
-        if (!__any_sync(FULL_MASK, joins && !(sum[R - 1] == old_tail))) break;
-    }
-    __syncwarp();  // every lane has read its products: s_val is free for the output
+        __syncwarp();  // every lane has read its products: the buffer is free for the output
 
-    // the last element of each run is emitted
-    const Key nextj = __shfl_down_sync(FULL_MASK, firstj, 1);
-    const bool next_valid = __shfl_down_sync(FULL_MASK, key[0] != PAD ? 1 : 0, 1) != 0 && lane < 31;
-    int ntails = 0;
-    bool tail[R];
+        // the last element of each run is emitted; element e = lane * R + r is real iff e < w
+        const int nreal = (int)w_n - lane * R;
+        int ntails = 0;
+        bool tail[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const bool same_next = (r + 1 < R) ? (key[r + 1] != PAD && (key[r + 1] >> IDXB) == (key[r] >> IDXB))
-                                           : (next_valid && nextj == (key[r] >> IDXB));
-        tail[r] = key[r] != PAD && !same_next;
-        ntails += tail[r];
-    }
-    const int tincl = warp_inclusive_scan(ntails);
-    const int total = __shfl_sync(FULL_MASK, tincl, 31);
-    int pos = tincl - ntails;
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        if (tail[r]) {
-            s_oj[warp][pos] = (int32_t)(key[r] >> IDXB);
-            s_val[warp][pos] = sum[r];
-            ++pos;
+        for (int r = 0; r < R; ++r) {
+            tail[r] = r < nreal && !(same[r + 1] && r + 1 < nreal);
+            ntails += tail[r];
         }
+        const int tincl = warp_inclusive_scan(ntails);
+        const int total = __shfl_sync(FULL_MASK, tincl, 31);
+        int pos = tincl - ntails;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if (tail[r]) {
+                s_j[warp][b][pos + (pos >> 3)] = (uint32_t)(key[r] >> IDXB);
+                s_v[warp][b][pos + (pos >> 3)] = sum[r];
+                ++pos;
+            }
+        }
+        __syncwarp();
+        for (int o = lane; o < total; o += 32) {
+            c_colidx[ob_n + o] = (int32_t)s_j[warp][b][o + (o >> 3)];
+            c_vals[ob_n + o] = (V)s_v[warp][b][o + (o >> 3)];
+        }
+        __syncwarp();  // buffer b is handed to the gathers of row n+2 in the next iteration
+
+        rloc_n = hB.x; w_n = w_next; ob_n = ob_next;
+        hB = hA; dB = dNew; aB = aNew; hA = hNew;
     }
-    __syncwarp();
-    const int64_t ob = c_rowptr[rloc];
-    for (int o = lane; o < total; o += 32) {
-        c_colidx[ob + o] = s_oj[warp][o];
-        c_vals[ob + o] = (V)s_val[warp][o];
-    }
+    cp_async_wait<0>();
+    (void)rloc_n;
 }
 
 }  // namespace spsyrk
