@@ -137,6 +137,38 @@ spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
                               void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
 
 /*
+ * spsyrk_mirror_rowptr_noalloc - the size step of spsyrk_mirror (step 2: d_f_rowptr[m + 1] and
+ * *nnz_full_out of F = C_L + C_L^T - D) for callers that can neither allocate device memory nor
+ * pass a workspace.  (The paper has no counterpart: this entry point exists for deployment only.)
+ *
+ * Who needs it: code that runs where device allocation is off limits - for instance a plug-in
+ * inside a host application that has reserved the whole GPU for its own memory pool, or a service
+ * loop that must not risk the device-wide synchronisation an allocation or a free can cause - and
+ * that therefore has no scratch buffer to hand to spsyrk_mirror.
+ *
+ * How: the scratch (two 32-bit counters per row, the scan's partial sums, an error word) is a
+ * fixed array inside the library image, SPSYRK_NOALLOC_MAX_ROWS rows long.  Every GPU that loads
+ * the library keeps those bytes (about 8 * SPSYRK_NOALLOC_MAX_ROWS) until the process exits.
+ * The call itself performs no cudaMalloc, cudaFree or any allocating library routine; the caller
+ * still owns and passes d_l_rowptr[m + 1], d_l_colidx[nnz_l] and d_f_rowptr[m + 1] (device) and
+ * nnz_full_out (host).
+ *
+ * Rules:
+ *   - m > SPSYRK_NOALLOC_MAX_ROWS is rejected with SPSYRK_ERR_OVERFLOW; use spsyrk_mirror then.
+ *   - The first call on a device looks up the array's device address (a one-time set-up per
+ *     device, done with that device current); make that first call before any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents; the
+ *     entry point clears what it accumulates into at the start of each call.  Two calls whose GPU
+ *     work overlaps in time (different streams or threads) race on it: serialise them.
+ *   - Synchronises the stream once (the entry count and the error word travel back).
+ * Results are identical to step 2 of spsyrk_mirror.
+ * Errors: INVALID_ARG, OVERFLOW, BAD_CSR (an entry above the diagonal), CUDA.
+ */
+#define SPSYRK_NOALLOC_MAX_ROWS 1048576
+spsyrk_status_t spsyrk_mirror_rowptr_noalloc(int64_t m, const int64_t *d_l_rowptr, const int32_t *d_l_colidx,
+                                             int64_t *d_f_rowptr, int64_t *nnz_full_out, void *cuda_stream);
+
+/*
  * spsyrk_jaccard - Jaccard similarity of the rows of a binary A from intersection counts,
  *     J_ij = c_ij / (|a_i| + |a_j| - c_ij),   |a_i| = stored entries of row i of A,
  * for rows [row_begin, row_begin + rows) of an int32-valued C_L with a tile-local row pointer

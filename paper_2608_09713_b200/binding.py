@@ -39,6 +39,8 @@ _lib.spsyrk_plan_set_rows.argtypes = [_vp, _i64, _i64, _vp]
 _lib.spsyrk_symbolic.argtypes = [_vp, _vp, _i64p, _vp]
 _lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
+_lib.spsyrk_mirror_rowptr_noalloc.argtypes = [_i64, _vp, _vp, _vp, _i64p, _vp]
+_lib.spsyrk_mirror_rowptr_noalloc.restype = _int
 _lib.spsyrk_jaccard.argtypes = [_i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_plan_stats.argtypes = [_vp, _i64p, _i64p]
 _lib.spsyrk_plan_buffers.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]
@@ -236,6 +238,22 @@ def spsyrk_mirror(m, l_rowptr, l_colidx, l_vals, stream=None, workspace=None):
     _check(_lib.spsyrk_mirror(m, nnz_l, code, _p(l_rowptr), _p(l_colidx), _p(l_vals), _p(f_rowptr), _p(f_colidx),
                               _p(f_vals), ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_mirror(fill)")
     return f_rowptr, f_colidx[:nnz.value], f_vals[:nnz.value]
+
+
+NOALLOC_MAX_ROWS = 1048576
+
+
+def spsyrk_mirror_rowptr_noalloc(m, l_rowptr, l_colidx, f_rowptr, stream=None) -> int:
+    """Row pointers of F = C_L + C_L^T - D into the caller's `f_rowptr` (m + 1 int64, CUDA) without
+    any device allocation and without a workspace: the library's built-in scratch array is used,
+    which caps m at NOALLOC_MAX_ROWS.  Returns nnz(F).  Calls that overlap on the GPU race on that
+    array; the first call on a device should precede any stream capture."""
+    _dev_check(l_rowptr, l_colidx, f_rowptr)
+    assert f_rowptr.dtype == torch.int64 and f_rowptr.numel() >= m + 1
+    nnz = ctypes.c_int64(0)
+    _check(_lib.spsyrk_mirror_rowptr_noalloc(m, _p(l_rowptr), _p(l_colidx), _p(f_rowptr), ctypes.byref(nnz),
+                                             _stream(stream)), "spsyrk_mirror_rowptr_noalloc")
+    return nnz.value
 
 
 def spsyrk_jaccard(m, row_begin, rows, a_rowptr, c_rowptr, c_colidx, c_counts, out=None, stream=None):

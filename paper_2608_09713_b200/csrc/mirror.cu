@@ -11,6 +11,7 @@
 //             behind the lower part: register bitonic sort for short segments, bitmap rank for
 //             long ones.
 #include <algorithm>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -314,4 +315,84 @@ extern "C" spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_
         case SPSYRK_F64: return mirror_fill<uint64_t>(w, m, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_f_rowptr, d_f_colidx, d_f_vals, st);
         default: return mirror_fill<uint32_t>(w, m, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_f_rowptr, d_f_colidx, d_f_vals, st);
     }
+}
+
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free variant of the size step of spsyrk_mirror.
+//
+// Some callers have no device memory to lend and may not create any: a plug-in running inside a
+// host application that has claimed the whole GPU for its own memory pool, or a service loop that
+// cannot afford the device-wide synchronisation a cudaMalloc / cudaFree may bring.  For them the
+// scratch of this one step lives in a fixed array that is part of the library image, so the call
+// needs nothing but its inputs and outputs.  The price: the array occupies its bytes on every GPU
+// that loads the library until the process exits, and the problem size is capped.
+// ------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int64_t NOALLOC_MAX_ROWS = SPSYRK_NOALLOC_MAX_ROWS;
+// strictly-lower counts (4 B per row), row totals (4 B per row), scan partials, one error word
+constexpr size_t NOALLOC_UCNT_OFF = 0;
+constexpr size_t NOALLOC_ROWTOT_OFF = NOALLOC_UCNT_OFF + (size_t)NOALLOC_MAX_ROWS * 4;
+constexpr size_t NOALLOC_PARTIALS_OFF = NOALLOC_ROWTOT_OFF + (size_t)NOALLOC_MAX_ROWS * 4;
+constexpr size_t NOALLOC_PARTIALS_BYTES = ((size_t)(NOALLOC_MAX_ROWS / SCAN_TILE) + 2) * 8;
+constexpr size_t NOALLOC_ERR_OFF = (NOALLOC_PARTIALS_OFF + NOALLOC_PARTIALS_BYTES + 255) / 256 * 256;
+constexpr size_t NOALLOC_BYTES = NOALLOC_ERR_OFF + 256;
+
+// In host code this name is only a handle for the runtime, not a device address: the address is
+// looked up once per device with cudaGetSymbolAddress and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+std::mutex g_noalloc_mutex;
+unsigned char* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
+
+// device address of the scratch array on the current device (set up on the first call per device)
+cudaError_t noalloc_scratch(unsigned char** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" spsyrk_status_t spsyrk_mirror_rowptr_noalloc(int64_t m, const int64_t* d_l_rowptr, const int32_t* d_l_colidx,
+                                                        int64_t* d_f_rowptr, int64_t* nnz_full_out, void* cuda_stream) {
+    if (m < 0 || !d_l_rowptr || !d_f_rowptr || !nnz_full_out) return SPSYRK_ERR_INVALID_ARG;
+    if (m > NOALLOC_MAX_ROWS) return SPSYRK_ERR_OVERFLOW;  // beyond the fixed scratch: use spsyrk_mirror
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    unsigned char* base = nullptr;
+    SPSYRK_CUDA_TRY(noalloc_scratch(&base));
+    uint32_t* ucnt = reinterpret_cast<uint32_t*>(base + NOALLOC_UCNT_OFF);
+    uint32_t* rowtot = reinterpret_cast<uint32_t*>(base + NOALLOC_ROWTOT_OFF);
+    int64_t* partials = reinterpret_cast<int64_t*>(base + NOALLOC_PARTIALS_OFF);
+    uint32_t* err = reinterpret_cast<uint32_t*>(base + NOALLOC_ERR_OFF);
+    // the array keeps whatever the previous call left: clear what is accumulated into
+    SPSYRK_CUDA_TRY(cudaMemsetAsync(err, 0, 4, st));
+    if (m > 0) {
+        SPSYRK_CUDA_TRY(cudaMemsetAsync(ucnt, 0, (size_t)m * 4, st));
+        // row lengths are not known on the host here, so the widest lane grouping is used
+        mirror_count_kernel<32><<<(unsigned)((m * 32 + 255) / 256), 256, 0, st>>>(d_l_rowptr, d_l_colidx, m, ucnt, err);
+        mirror_rowtot_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(d_l_rowptr, ucnt, m, rowtot);
+        note_launches(2);
+    }
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(rowtot, m, d_f_rowptr, partials, st));
+    int64_t nnz = 0;
+    uint32_t e = 0;
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(&nnz, d_f_rowptr + m, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(&e, err, 4, cudaMemcpyDeviceToHost, st));
+    SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
+    if (e & ERRW_UPPER) return SPSYRK_ERR_BAD_CSR;
+    *nnz_full_out = nnz;
+    return SPSYRK_OK;
 }
