@@ -1,0 +1,116 @@
+"""The five benchmark configurations at full size, in the launch configuration bench.py times
+(one plan over all rows, TRIL): sampled output rows against the CPU oracle, plus properties that
+hold at any size (closed-form counts, diagonal = squared row norms, the sum identity, mirror and
+Jaccard invariants)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_09713_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TOL = {np.dtype(np.float64): 1e-12, np.dtype(np.float32): 1e-5}
+
+
+@pytest.fixture(scope="module")
+def B():
+    assert torch.cuda.is_available()
+    from paper_2608_09713_b200 import binding
+    return binding
+
+
+def sample_rows(m, deg, k, seed):
+    rng = np.random.default_rng(seed)
+    rows = set(rng.integers(0, m, size=k).tolist()) | {0, 1, m // 2, m - 2, m - 1}
+    heavy = np.argsort(deg)[-3:]                       # the heaviest rows of A as well
+    return sorted(rows | set(int(x) for x in heavy))
+
+
+def check_rows_against_oracle(a, cols, mode, rows, rp, ci, cv):
+    for r in rows:
+        ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, mode, r, r + 1, cols=cols)
+        lo, hi = int(rp[r]), int(rp[r + 1])
+        assert hi - lo == ref.nnz, f"row {r}: count"
+        got_c = ci[lo:hi].cpu().numpy()
+        got_v = cv[lo:hi].cpu().numpy()
+        assert np.array_equal(got_c, ref.colidx), f"row {r}: structure"
+        if np.issubdtype(a.vals.dtype, np.integer):
+            assert np.array_equal(got_v, oracle.to_int32(ref.vals)), f"row {r}: values"
+        else:
+            err = np.abs(got_v.astype(np.float64) - ref.vals)
+            assert np.all(err <= TOL[np.dtype(a.vals.dtype)] * ref.absvals), f"row {r}: values"
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_full_size_configuration(B, idx):
+    a = W.config(idx)
+    deg = np.diff(a.rowptr)
+    d = (torch.from_numpy(a.rowptr).cuda(), torch.from_numpy(a.colidx).cuda(), torch.from_numpy(a.vals).cuda())
+    rp, ci, cv, plan = B.tril_syrk(a.m, a.n, *d)
+    torch.cuda.synchronize()
+    rp_h = rp.cpu().numpy()
+    nnz = int(rp_h[-1])
+
+    # closed forms: multiply-add count of the half (Section III-C restricted to pairs j <= i)
+    dk = np.bincount(a.colidx, minlength=a.n).astype(np.int64)
+    work, classes = B.spsyrk_plan_stats(plan)
+    assert work == int((dk * (dk + 1) // 2).sum())
+    assert sum(classes) == a.m
+    cnt = np.diff(rp_h)
+    assert np.array_equal(cnt >= 1, deg > 0) and np.all(cnt <= np.arange(a.m) + 1)
+    if idx == 2:
+        assert dk.max() == a.m and nnz == a.m * (a.m + 1) // 2          # a column in every row: dense output
+
+    # the diagonal is the last entry of every non-empty row and equals the squared row norm
+    last = rp[1:][torch.from_numpy(deg > 0).cuda()] - 1
+    rows_ne = torch.from_numpy(np.nonzero(deg > 0)[0]).cuda()
+    assert torch.equal(ci[last].to(torch.int64), rows_ne)
+    sq = torch.zeros(a.m, dtype=torch.float64, device="cuda")
+    sq.index_add_(0, torch.repeat_interleave(torch.arange(a.m, device="cuda"), torch.from_numpy(deg).cuda()),
+                  d[2].to(torch.float64) ** 2)
+    diag = cv[last].to(torch.float64)
+    tol = 1e-5 if a.vals.dtype == np.float32 else 1e-12
+    assert torch.all((diag - sq[rows_ne]).abs() <= tol * sq[rows_ne])
+
+    # sum identity: 2 sum(C_L) - trace = sum_k (sum_i a_ik)^2
+    colsum = np.zeros(a.n)
+    np.add.at(colsum, a.colidx, a.vals.astype(np.float64))
+    abssum = np.zeros(a.n)
+    np.add.at(abssum, a.colidx, np.abs(a.vals.astype(np.float64)))
+    if a.vals.dtype == np.int32:
+        lhs = 2 * int(cv.sum(dtype=torch.int64).item()) - int(diag.sum().item())
+        assert lhs == int((colsum ** 2).sum())
+    else:
+        lhs = 2 * float(cv.to(torch.float64).sum().item()) - float(diag.sum().item())
+        assert abs(lhs - (colsum ** 2).sum()) <= (1e-4 if a.vals.dtype == np.float32 else 1e-9) * (abssum ** 2).sum()
+
+    # sampled rows against the oracle
+    cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
+    rows = sample_rows(a.m, deg, 12 if idx == 2 else 40, idx)
+    check_rows_against_oracle(a, cols, oracle.TRIL, rows, rp_h, ci, cv)
+
+    # Jaccard on the binary configuration
+    if a.vals.dtype == np.int32:
+        jac = B.spsyrk_jaccard(a.m, 0, a.m, d[0], rp, ci, cv)
+        assert torch.all(jac[last] == 1.0)
+        for r in rows[:6]:
+            lo, hi = int(rp_h[r]), int(rp_h[r + 1])
+            exp = oracle.jaccard(r, 1, a.rowptr, np.array([0, hi - lo]), ci[lo:hi].cpu().numpy(), cv[lo:hi].cpu().numpy())
+            assert np.array_equal(jac[lo:hi].cpu().numpy(), exp)
+        del jac
+
+    # mirror on the configurations that ask for it (4 and 5) and on the small ones
+    if idx in (1, 3, 4, 5):
+        f_rowptr, f_colidx, f_vals = B.spsyrk_mirror(a.m, rp, ci, cv)
+        torch.cuda.synchronize()
+        frp = f_rowptr.cpu().numpy()
+        assert int(frp[-1]) == 2 * nnz - int((deg > 0).sum())
+        # rows of F are rows of the full product: same structure, values within the tolerance
+        check_rows_against_oracle(a, cols, oracle.FULL, rows[:20], frp, f_colidx, f_vals)
+        # lower parts are bit copies of C_L
+        for r in rows[:20]:
+            lo, hi = int(rp_h[r]), int(rp_h[r + 1])
+            assert torch.equal(f_colidx[int(frp[r]):int(frp[r]) + hi - lo], ci[lo:hi])
+            assert torch.equal(f_vals[int(frp[r]):int(frp[r]) + hi - lo], cv[lo:hi])
