@@ -126,8 +126,7 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t *d_c_rowptr,
  * Three-step use:
  *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for (m, nnz_l, dtype).
  *   2. d_f_colidx == NULL: writes d_f_rowptr[m + 1] and *nnz_full_out (synchronises).
- *   3. all pointers set: fills d_f_colidx / d_f_vals using the d_f_rowptr of step 2 (synchronises once,
- *      to size the per-class launches of its segment sort).
+ *   3. all pointers set: fills d_f_colidx / d_f_vals using the d_f_rowptr of step 2.  Asynchronous.
  * nnz_l = d_l_rowptr[m].  Errors: INVALID_ARG, WORKSPACE, BAD_CSR (an entry above the diagonal), CUDA.
  */
 spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,

@@ -2,38 +2,38 @@
 //
 // Row j of F = row j of C_L (columns <= j) followed by the reflected entries (r, c_rj) of the
 // later rows r > j that store column j, ascending in r.  That second part is a transpose of the
-// strictly lower triangle:
+// strictly lower triangle, done as a stable radix sort of the entries by column id:
 //   count   : per column j the number of strictly lower entries (atomics), add the row's own
 //             length, scan -> f_rowptr.
-//   scatter : copy the lower parts in place; push every strictly lower entry (r, j, v) into the
-//             staging segment of row j through an atomic cursor (arbitrary order inside a segment).
-//   sort    : order every staging segment by r (rows are distinct inside a segment) and write it
-//             behind the lower part: register bitonic sort for short segments, bitmap rank for
-//             long ones.
+//   expand  : copy the lower parts into F; write an explicit (key, row) pair per entry, the key
+//             being the column id, or m for a diagonal entry so that diagonals sort past the end.
+//   sort    : stable LSD radix passes over (key, row, value); entries enter in ascending row order,
+//             so every column's segment comes out ascending in r.  The last pass writes straight
+//             into F: the s-th strictly lower entry in sorted order, of column j, lands at
+//             s + l_rowptr[j + 1].
 #include <algorithm>
 #include <mutex>
 
-#include "common.cuh"
+#include "radix.cuh"
 
 using namespace spsyrk;
 
 namespace {
 
 constexpr size_t ALIGN = 256;
-constexpr uint32_t MIRROR_CHUNK_BITS_MAX = 1u << 19;
+
+constexpr int MIRROR_RADIX_BITS = 8;
 
 struct MirrorWs {
-    uint32_t* ucnt;    // m: strictly-lower entries per column, later reused as cursor
+    uint32_t* ucnt;    // m: strictly-lower entries per column
     uint32_t* rowtot;  // m
-    uint8_t* cls;      // m
-    int32_t* perm;     // m
-    int32_t* blockhist;
-    int64_t* offsets;
     int64_t* partials;
-    int64_t* class_start_dev;
     uint32_t* err;
-    int32_t* stage_row;  // nnz_l
-    void* stage_val;     // nnz_l * sv
+    // radix sort buffers (nnz_l entries each); buffer B's key and row arrays double as the expanded input
+    uint32_t *key_a, *row_a, *key_b, *row_b;
+    void *val_a, *val_b;
+    uint32_t* hist;
+    int64_t* offsets;
 };
 
 size_t carve(MirrorWs* w, void* ws, int64_t m, int64_t nnz_l, size_t sv) {
@@ -46,19 +46,21 @@ size_t carve(MirrorWs* w, void* ws, int64_t m, int64_t nnz_l, size_t sv) {
         return p;
     };
     const int64_t items = std::max<int64_t>(m, 1);
-    const int64_t nb = bin_blocks(items);
+    const int64_t ne = std::max<int64_t>(nnz_l, 1);
+    const int64_t hist_n = (int64_t)(1 << MIRROR_RADIX_BITS) * std::max<int64_t>(radix_tiles(nnz_l), 1);
     MirrorWs t;
     t.ucnt = (uint32_t*)take(items * 4);
     t.rowtot = (uint32_t*)take(items * 4);
-    t.cls = (uint8_t*)take(items);
-    t.perm = (int32_t*)take(items * 4);
-    t.blockhist = (int32_t*)take(NCLASS * nb * 4);
-    t.offsets = (int64_t*)take((NCLASS * nb + 1) * 8);
-    t.partials = (int64_t*)take(scan_partials_count(std::max<int64_t>(items + 1, NCLASS * nb)) * 8);
-    t.class_start_dev = (int64_t*)take((NCLASS + 1) * 8);
+    t.partials = (int64_t*)take(scan_partials_count(std::max<int64_t>(items + 1, hist_n)) * 8);
     t.err = (uint32_t*)take(4);
-    t.stage_row = (int32_t*)take(std::max<int64_t>(nnz_l, 1) * 4);
-    t.stage_val = take(std::max<int64_t>(nnz_l, 1) * sv);
+    t.key_a = (uint32_t*)take(ne * 4);
+    t.row_a = (uint32_t*)take(ne * 4);
+    t.key_b = (uint32_t*)take(ne * 4);
+    t.row_b = (uint32_t*)take(ne * 4);
+    t.val_a = take(ne * sv);
+    t.val_b = take(ne * sv);
+    t.hist = (uint32_t*)take(hist_n * 4);
+    t.offsets = (int64_t*)take((hist_n + 1) * 8);
     if (w) *w = t;
     return (off + ALIGN - 1) / ALIGN * ALIGN;
 }
@@ -83,21 +85,13 @@ __global__ void mirror_rowtot_kernel(const int64_t* __restrict__ l_rowptr, const
     if (r < m) rowtot[r] = (uint32_t)(l_rowptr[r + 1] - l_rowptr[r]) + ucnt[r];
 }
 
-// class of a row of F by the length u of its reflected part
-__global__ void mirror_class_kernel(const int64_t* __restrict__ l_rowptr, const int64_t* __restrict__ f_rowptr, int64_t m,
-                                    uint8_t* __restrict__ cls) {
-    int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= m) return;
-    const int64_t u = (f_rowptr[r + 1] - f_rowptr[r]) - (l_rowptr[r + 1] - l_rowptr[r]);
-    cls[r] = u <= 0 ? 0 : u <= 32 ? 1 : u <= 64 ? 2 : u <= 128 ? 3 : u <= 256 ? 4 : u <= 512 ? 5 : 7;
-}
-
+// G lanes per row: copy the row into F and write the explicit (key, row) pair of every entry.
 template <typename V, int G>
-__global__ void __launch_bounds__(256) mirror_scatter_kernel(const int64_t* __restrict__ l_rowptr, const int32_t* __restrict__ l_colidx,
-                                                             const V* __restrict__ l_vals, int64_t m,
-                                                             const int64_t* __restrict__ f_rowptr, int32_t* __restrict__ f_colidx,
-                                                             V* __restrict__ f_vals, uint32_t* __restrict__ cursor,
-                                                             int32_t* __restrict__ stage_row, V* __restrict__ stage_val) {
+__global__ void __launch_bounds__(256) mirror_expand_kernel(const int64_t* __restrict__ l_rowptr, const int32_t* __restrict__ l_colidx,
+                                                            const V* __restrict__ l_vals, int64_t m,
+                                                            const int64_t* __restrict__ f_rowptr, int32_t* __restrict__ f_colidx,
+                                                            V* __restrict__ f_vals, uint32_t* __restrict__ key0,
+                                                            uint32_t* __restrict__ row0) {
     const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
     const int gl = threadIdx.x & (G - 1);
     if (r >= m) return;
@@ -105,158 +99,71 @@ __global__ void __launch_bounds__(256) mirror_scatter_kernel(const int64_t* __re
     const int64_t fb = f_rowptr[r];
     for (int64_t p = p0 + gl; p < p1; p += G) {
         const int32_t j = l_colidx[p];
-        const V v = l_vals[p];
         f_colidx[fb + (p - p0)] = j;
-        f_vals[fb + (p - p0)] = v;
-        if (j < r) {
-            const uint32_t slot = atomicAdd(&cursor[j], 1u);
-            const int64_t sp = (f_rowptr[j] - l_rowptr[j]) + slot;  // segment start = reflected entries of earlier rows
-            stage_row[sp] = (int32_t)r;
-            stage_val[sp] = v;
-        }
+        f_vals[fb + (p - p0)] = l_vals[p];
+        key0[p] = j == r ? (uint32_t)m : (uint32_t)j;
+        row0[p] = (uint32_t)r;
     }
 }
 
-// one warp per row of F whose reflected part has at most 32*R entries
-template <typename V, int R, typename Key>
-__global__ void __launch_bounds__(256) mirror_sort_warp_kernel(const int32_t* __restrict__ rows, int64_t nrows,
-                                                               const int64_t* __restrict__ l_rowptr, const int64_t* __restrict__ f_rowptr,
-                                                               const int32_t* __restrict__ stage_row, const V* __restrict__ stage_val,
-                                                               int32_t* __restrict__ f_colidx, V* __restrict__ f_vals) {
-    constexpr int IDXB = ilog2_ce(32 * R);
-    const int lane = lane_id();
-    const int64_t widx = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (widx >= nrows) return;
-    const int64_t j = rows[widx];
-    const int64_t lcnt = l_rowptr[j + 1] - l_rowptr[j];
-    const int64_t sb = f_rowptr[j] - l_rowptr[j];
-    const int64_t fb = f_rowptr[j] + lcnt;
-    const uint32_t u = (uint32_t)(f_rowptr[j + 1] - fb);
-    Key x[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const uint32_t e = r * 32 + lane;
-        x[r] = e < u ? (((Key)(uint32_t)stage_row[sb + e] << IDXB) | (Key)e) : ~Key(0);
-    }
-    group_bitonic_sort<Key, R, 32>(x);
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const uint32_t q = lane * R + r;
-        if (q < u) {
-            f_colidx[fb + q] = (int32_t)(x[r] >> IDXB);
-            f_vals[fb + q] = stage_val[sb + (uint32_t)(x[r] & (Key)(32 * R - 1))];
+template <typename V>
+struct EmitMirrorFinal {
+    const int64_t* l_rowptr;
+    int32_t* f_colidx;
+    V* f_vals;
+    uint32_t m;
+    __device__ __forceinline__ void operator()(int64_t dest, uint32_t key, uint32_t row, V val) const {
+        if (key < m) {  // diagonal entries were keyed m and are dropped here
+            const int64_t pos = dest + l_rowptr[key + 1];
+            f_colidx[pos] = (int32_t)row;
+            f_vals[pos] = val;
         }
     }
-}
-
-// one CTA per row of F with a long reflected part: bitmap rank over chunks of the row-id range (j, m)
-template <typename V, int THREADS>
-__global__ void __launch_bounds__(THREADS) mirror_sort_cta_kernel(const int32_t* __restrict__ rows, int64_t m, uint32_t chunk_bits,
-                                                                  const int64_t* __restrict__ l_rowptr, const int64_t* __restrict__ f_rowptr,
-                                                                  const int32_t* __restrict__ stage_row, const V* __restrict__ stage_val,
-                                                                  int32_t* __restrict__ f_colidx, V* __restrict__ f_vals) {
-    extern __shared__ uint32_t smem_u32[];
-    __shared__ uint32_t scratch[33];
-    const uint32_t cw = chunk_bits >> 5;
-    uint32_t* bits = smem_u32;
-    uint32_t* rank = smem_u32 + cw;
-    const int64_t j = rows[blockIdx.x];
-    const int64_t lcnt = l_rowptr[j + 1] - l_rowptr[j];
-    const int64_t sb = f_rowptr[j] - l_rowptr[j];
-    const int64_t fb = f_rowptr[j] + lcnt;
-    const uint32_t u = (uint32_t)(f_rowptr[j + 1] - fb);
-    const uint32_t per = (cw + THREADS - 1) / THREADS;
-    uint32_t base = 0;
-    for (int64_t c0 = j + 1; c0 < m; c0 += chunk_bits) {
-        for (uint32_t w = threadIdx.x; w < cw; w += THREADS) bits[w] = 0;
-        __syncthreads();
-        for (uint32_t e = threadIdx.x; e < u; e += THREADS) {
-            const int64_t rel = (int64_t)stage_row[sb + e] - c0;
-            if (rel >= 0 && rel < (int64_t)chunk_bits) atomicOr(&bits[rel >> 5], 1u << (rel & 31));
-        }
-        __syncthreads();
-        uint32_t s = 0;
-        const uint32_t w0 = threadIdx.x * per;
-        for (uint32_t w = w0; w < w0 + per && w < cw; ++w) s += __popc(bits[w]);
-        uint32_t tot;
-        uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(s, scratch, &tot);
-        for (uint32_t w = w0; w < w0 + per && w < cw; ++w) { rank[w] = ex; ex += __popc(bits[w]); }
-        __syncthreads();
-        for (uint32_t e = threadIdx.x; e < u; e += THREADS) {
-            const int32_t r = stage_row[sb + e];
-            const int64_t rel = (int64_t)r - c0;
-            if (rel >= 0 && rel < (int64_t)chunk_bits) {
-                const uint32_t q = base + rank[rel >> 5] + __popc(bits[rel >> 5] & ((1u << (rel & 31)) - 1u));
-                f_colidx[fb + q] = r;
-                f_vals[fb + q] = stage_val[sb + e];
-            }
-        }
-        base += tot;
-        __syncthreads();
-    }
-}
+};
 
 int group_width(int64_t nnz, int64_t m) {
     const double avg = m > 0 ? (double)nnz / (double)m : 0.0;
     return avg <= 4 ? 4 : avg <= 8 ? 8 : avg <= 16 ? 16 : 32;
 }
 
-template <typename V, int R, typename Key>
-void launch_sort_warp(const MirrorWs& w, const int64_t* cs, int c, const int64_t* l_rowptr, const int64_t* f_rowptr,
-                      int32_t* f_colidx, void* f_vals, cudaStream_t st) {
-    const int64_t count = cs[c + 1] - cs[c];
-    if (count <= 0) return;
-    mirror_sort_warp_kernel<V, R, Key><<<(unsigned)((count * 32 + 255) / 256), 256, 0, st>>>(
-        w.perm + cs[c], count, l_rowptr, f_rowptr, w.stage_row, static_cast<const V*>(w.stage_val), f_colidx, static_cast<V*>(f_vals));
-    note_launches(1);
-}
-
-template <typename V, typename Key>
-void launch_sort_warp_all(const MirrorWs& w, const int64_t* cs, const int64_t* l_rowptr, const int64_t* f_rowptr,
-                          int32_t* f_colidx, void* f_vals, cudaStream_t st) {
-    launch_sort_warp<V, 1, Key>(w, cs, 1, l_rowptr, f_rowptr, f_colidx, f_vals, st);
-    launch_sort_warp<V, 2, Key>(w, cs, 2, l_rowptr, f_rowptr, f_colidx, f_vals, st);
-    launch_sort_warp<V, 4, Key>(w, cs, 3, l_rowptr, f_rowptr, f_colidx, f_vals, st);
-    launch_sort_warp<V, 8, Key>(w, cs, 4, l_rowptr, f_rowptr, f_colidx, f_vals, st);
-    launch_sort_warp<V, 16, Key>(w, cs, 5, l_rowptr, f_rowptr, f_colidx, f_vals, st);
-}
-
 template <typename V>
 spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const int64_t* l_rowptr, const int32_t* l_colidx,
                             const void* l_vals, const int64_t* f_rowptr, int32_t* f_colidx, void* f_vals, cudaStream_t st) {
-    SPSYRK_CUDA_TRY(cudaMemsetAsync(w.ucnt, 0, (size_t)m * 4, st));
+    constexpr int BITS = MIRROR_RADIX_BITS;
     const V* lv = static_cast<const V*>(l_vals);
     V* fv = static_cast<V*>(f_vals);
-    V* sv = static_cast<V*>(w.stage_val);
-#define SCATTER(G)                                                                                                   \
-    mirror_scatter_kernel<V, G><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(l_rowptr, l_colidx, lv, m, f_rowptr, \
-                                                                                 f_colidx, fv, w.ucnt, w.stage_row, sv)
+#define EXPAND(G)                                                                                                   \
+    mirror_expand_kernel<V, G><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(l_rowptr, l_colidx, lv, m, f_rowptr, \
+                                                                                f_colidx, fv, w.key_b, w.row_b)
     switch (group_width(nnz_l, m)) {
-        case 4: SCATTER(4); break;
-        case 8: SCATTER(8); break;
-        case 16: SCATTER(16); break;
-        default: SCATTER(32); break;
+        case 4: EXPAND(4); break;
+        case 8: EXPAND(8); break;
+        case 16: EXPAND(16); break;
+        default: EXPAND(32); break;
     }
-#undef SCATTER
-    mirror_class_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(l_rowptr, f_rowptr, m, w.cls);
-    note_launches(2);  // scatter + class
-    SPSYRK_CUDA_TRY(bin_items(w.cls, m, w.perm, w.class_start_dev, w.blockhist, w.offsets, w.partials, st));
-    int64_t cs[NCLASS + 1];
-    SPSYRK_CUDA_TRY(cudaMemcpyAsync(cs, w.class_start_dev, sizeof(cs), cudaMemcpyDeviceToHost, st));
-    SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
-    if (m <= (int64_t(1) << 22)) launch_sort_warp_all<V, uint32_t>(w, cs, l_rowptr, f_rowptr, f_colidx, f_vals, st);
-    else launch_sort_warp_all<V, uint64_t>(w, cs, l_rowptr, f_rowptr, f_colidx, f_vals, st);
-    const int64_t big = cs[8] - cs[7];
-    if (big > 0) {
-        uint32_t cb = 1024;
-        while (cb < MIRROR_CHUNK_BITS_MAX && cb < (uint64_t)m) cb <<= 1;
-        const size_t smem = (size_t)(cb >> 5) * 2 * sizeof(uint32_t);
-        auto kern = mirror_sort_cta_kernel<V, 512>;
-        SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<(unsigned)big, 512, smem, st>>>(w.perm + cs[7], m, cb, l_rowptr, f_rowptr, w.stage_row, sv, f_colidx, fv);
-        note_launches(1);
+#undef EXPAND
+    note_launches(1);
+    if (nnz_l == 0) return SPSYRK_OK;
+    const int npass = (bits_for((uint64_t)m) + BITS - 1) / BITS;  // keys run from 0 to m
+    const uint32_t* src_key = w.key_b;
+    const uint32_t* src_row = w.row_b;
+    const V* src_val = lv;
+    for (int p = 0; p < npass; ++p) {
+        const bool to_a = (p % 2) == 0;
+        uint32_t* dst_key = to_a ? w.key_a : w.key_b;
+        uint32_t* dst_row = to_a ? w.row_a : w.row_b;
+        V* dst_val = static_cast<V*>(to_a ? w.val_a : w.val_b);
+        if (p == npass - 1) {
+            EmitMirrorFinal<V> emit{l_rowptr, f_colidx, fv, (uint32_t)m};
+            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+        } else {
+            EmitArrays<V> emit{dst_key, dst_row, dst_val};
+            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+        }
+        src_key = dst_key;
+        src_row = dst_row;
+        src_val = dst_val;
     }
-    SPSYRK_CUDA_TRY(cudaGetLastError());
     return SPSYRK_OK;
 }
 
