@@ -74,7 +74,7 @@ typedef enum { SPSYRK_TRIL = 0, SPSYRK_FULL = 1 } spsyrk_mode_t;
  * Row tiles: plans for disjoint row ranges are independent; concatenating their results gives
  * the untiled C_L.  (Halving a CSR matrix along rows is free, Section IV-A.)
  *
- * d_rowptr[m+1], d_colidx[nnz], d_vals[nnz] of `dtype`.  0 <= row_begin <= row_end <= m.
+ * d_rowptr[m+1], d_colidx[nnz] (16-byte aligned), d_vals[nnz] of `dtype`.  0 <= row_begin <= row_end <= m.
  * Errors: INVALID_ARG, OVERFLOW, WORKSPACE, BAD_CSR, CUDA.
  */
 spsyrk_status_t spsyrk_plan(spsyrk_plan_t *plan, int64_t m, int64_t n, int64_t nnz,
@@ -127,7 +127,7 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t *d_c_rowptr,
  *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for (m, nnz_l, dtype).
  *   2. d_f_colidx == NULL: writes d_f_rowptr[m + 1] and *nnz_full_out (synchronises).
  *   3. all pointers set: fills d_f_colidx / d_f_vals using the d_f_rowptr of step 2.  Asynchronous.
- * nnz_l = d_l_rowptr[m].  Errors: INVALID_ARG, WORKSPACE, BAD_CSR (an entry above the diagonal), CUDA.
+ * nnz_l = d_l_rowptr[m].  d_l_vals must be 16-byte aligned.  Errors: INVALID_ARG, WORKSPACE, BAD_CSR (an entry above the diagonal), CUDA.
  */
 spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
                               const int64_t *d_l_rowptr, const int32_t *d_l_colidx, const void *d_l_vals,

@@ -123,7 +123,7 @@ def spsyrk_plan_workspace_bytes(m, n, nnz, dtype=torch.float64, mode=TRIL) -> in
     return sz.value
 
 
-def spsyrk_plan(m, n, rowptr, colidx, vals, mode=TRIL, row_begin=0, row_end=None, stream=None) -> Plan:
+def spsyrk_plan(m, n, rowptr, colidx, vals, mode=TRIL, row_begin=0, row_end=None, stream=None, workspace=None) -> Plan:
     _dev_check(rowptr, colidx, vals)
     assert rowptr.dtype == torch.int64 and colidx.dtype == torch.int32 and vals.dtype in _DTYPE_CODE
     row_end = m if row_end is None else row_end
@@ -132,7 +132,9 @@ def spsyrk_plan(m, n, rowptr, colidx, vals, mode=TRIL, row_begin=0, row_end=None
     sz = ctypes.c_size_t(0)
     _check(_lib.spsyrk_plan(None, m, n, nnz, None, None, None, code, mode, row_begin, row_end, None,
                             ctypes.byref(sz), None), "spsyrk_plan(size query)")
-    ws = _workspace(sz.value, rowptr.device)
+    ws = workspace if workspace is not None else _workspace(sz.value, rowptr.device)
+    assert ws.numel() >= sz.value
+    sz = ctypes.c_size_t(ws.numel())
     h = _vp()
     _check(_lib.spsyrk_plan(ctypes.byref(h), m, n, nnz, _p(rowptr), _p(colidx), _p(vals), code, mode, row_begin,
                             row_end, _p(ws), ctypes.byref(sz), _stream(stream)), "spsyrk_plan")
@@ -219,8 +221,9 @@ def spsyrk_mirror_workspace_bytes(m, nnz_l, dtype) -> int:
     return sz.value
 
 
-def spsyrk_mirror(m, l_rowptr, l_colidx, l_vals, stream=None, workspace=None):
-    """Returns (f_rowptr, f_colidx, f_vals) of F = C_L + C_L^T - D; allocates the outputs with torch."""
+def spsyrk_mirror(m, l_rowptr, l_colidx, l_vals, stream=None, workspace=None, out=None):
+    """Returns (f_rowptr, f_colidx, f_vals) of F = C_L + C_L^T - D.  The outputs are allocated with torch
+    unless `out` = (f_rowptr, f_colidx, f_vals) supplies buffers that are large enough."""
     _dev_check(l_rowptr, l_colidx, l_vals)
     nnz_l = l_colidx.numel()
     code = _DTYPE_CODE[l_vals.dtype]
@@ -228,13 +231,17 @@ def spsyrk_mirror(m, l_rowptr, l_colidx, l_vals, stream=None, workspace=None):
     ws = workspace if workspace is not None else _workspace(sz.value, l_rowptr.device)
     assert ws.numel() >= sz.value
     sz = ctypes.c_size_t(ws.numel())
-    f_rowptr = torch.empty(m + 1, dtype=torch.int64, device=l_rowptr.device)
+    f_rowptr = out[0] if out is not None else torch.empty(m + 1, dtype=torch.int64, device=l_rowptr.device)
     nnz = ctypes.c_int64(0)
     st = _stream(stream)
     _check(_lib.spsyrk_mirror(m, nnz_l, code, _p(l_rowptr), _p(l_colidx), _p(l_vals), _p(f_rowptr), None, None,
                               ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_mirror(sizes)")
-    f_colidx = torch.empty(max(nnz.value, 1), dtype=torch.int32, device=l_rowptr.device)
-    f_vals = torch.empty(max(nnz.value, 1), dtype=l_vals.dtype, device=l_rowptr.device)
+    if out is not None:
+        f_colidx, f_vals = out[1], out[2]
+        assert f_colidx.numel() >= nnz.value and f_vals.numel() >= nnz.value and f_vals.dtype == l_vals.dtype
+    else:
+        f_colidx = torch.empty(max(nnz.value, 1), dtype=torch.int32, device=l_rowptr.device)
+        f_vals = torch.empty(max(nnz.value, 1), dtype=l_vals.dtype, device=l_rowptr.device)
     _check(_lib.spsyrk_mirror(m, nnz_l, code, _p(l_rowptr), _p(l_colidx), _p(l_vals), _p(f_rowptr), _p(f_colidx),
                               _p(f_vals), ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_mirror(fill)")
     return f_rowptr, f_colidx[:nnz.value], f_vals[:nnz.value]

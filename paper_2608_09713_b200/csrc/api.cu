@@ -22,7 +22,7 @@ constexpr size_t ALIGN = 256;
 constexpr int64_t BLOCK_CLASS_MAX_WORK = 16384;  // class 6 (256-thread CTA) up to here, class 7 above
 constexpr uint32_t ROW_CHUNK_BITS_MAX_NUMERIC = 1u << 18;
 constexpr uint32_t ROW_CHUNK_BITS_MAX_SYMBOLIC = 1u << 20;
-constexpr uint32_t COL_CHUNK_BITS_MAX = 1u << 19;
+constexpr int TRANSPOSE_RADIX_BITS = 8;
 constexpr size_t LARGE_SMEM_BUDGET = 200 * 1024;
 constexpr uint32_t BLOCK_ACC_SLOTS = 4096;
 
@@ -58,10 +58,11 @@ struct spsyrk_plan_s {
     uint4* hdr;  // per-row headers in class order
     int32_t* cnt;
     uint8_t* cls;
-    uint64_t* keys;
     uint32_t* colcnt;
-    uint32_t* cursor;
-    int32_t* colperm;
+    // radix sort buffers of the transpose (nnz entries each) and its histograms
+    uint32_t *rx_key_a, *rx_row_a, *rx_pos_a, *rx_key_b, *rx_row_b, *rx_pos_b;
+    uint32_t* rx_hist;
+    int64_t* rx_offsets;
     int32_t* blockhist;
     int64_t* offsets;
     int64_t* partials;
@@ -94,21 +95,29 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     auto hdr = c.take<uint4>(m);
     auto cnt = c.take<int32_t>(m);
     auto cls = c.take<uint8_t>(items);
-    auto keys = c.take<uint64_t>(nnz);
     auto colcnt = c.take<uint32_t>(n);
-    auto cursor = c.take<uint32_t>(n);
-    auto colperm = c.take<int32_t>(n);
+    const int64_t rx_hist_n = (int64_t)(1 << TRANSPOSE_RADIX_BITS) * std::max<int64_t>(radix_tiles(nnz), 1);
+    auto rx_key_a = c.take<uint32_t>(nnz);
+    auto rx_row_a = c.take<uint32_t>(nnz);
+    auto rx_pos_a = c.take<uint32_t>(nnz);
+    auto rx_key_b = c.take<uint32_t>(nnz);
+    auto rx_row_b = c.take<uint32_t>(nnz);
+    auto rx_pos_b = c.take<uint32_t>(nnz);
+    auto rx_hist = c.take<uint32_t>(rx_hist_n);
+    auto rx_offsets = c.take<int64_t>(rx_hist_n + 1);
     auto blockhist = c.take<int32_t>(NCLASS * nb);
     auto offsets = c.take<int64_t>(NCLASS * nb + 1);
-    auto partials = c.take<int64_t>(scan_partials_count(std::max<int64_t>(items + 1, NCLASS * nb)));
+    auto partials = c.take<int64_t>(scan_partials_count(std::max<int64_t>(std::max<int64_t>(items + 1, NCLASS * nb), rx_hist_n)));
     auto class_start_dev = c.take<int64_t>(NCLASS + 1);
     auto work_total_dev = c.take<unsigned long long>(1);
     auto err = c.take<uint32_t>(1);
     if (pl) {
         pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.desc = desc;
         pl->dev.work = work; pl->dev.err = err;
-        pl->perm = perm; pl->hdr = hdr; pl->cnt = cnt; pl->cls = cls; pl->keys = keys; pl->colcnt = colcnt; pl->cursor = cursor;
-        pl->colperm = colperm; pl->blockhist = blockhist; pl->offsets = offsets; pl->partials = partials;
+        pl->perm = perm; pl->hdr = hdr; pl->cnt = cnt; pl->cls = cls; pl->colcnt = colcnt;
+        pl->rx_key_a = rx_key_a; pl->rx_row_a = rx_row_a; pl->rx_pos_a = rx_pos_a; pl->rx_key_b = rx_key_b; pl->rx_row_b = rx_row_b;
+        pl->rx_pos_b = rx_pos_b; pl->rx_hist = rx_hist; pl->rx_offsets = rx_offsets;
+        pl->blockhist = blockhist; pl->offsets = offsets; pl->partials = partials;
         pl->class_start_dev = class_start_dev; pl->work_total_dev = work_total_dev;
     }
     return (c.off + ALIGN - 1) / ALIGN * ALIGN;
@@ -124,11 +133,10 @@ spsyrk_status_t read_err(spsyrk_plan_s* pl, cudaStream_t st) {
 }
 
 template <int G>
-void launch_fill(spsyrk_plan_s* pl, cudaStream_t st) {
+void launch_row_expand(spsyrk_plan_s* pl, cudaStream_t st) {
     const PlanDev& P = pl->dev;
     const int64_t threads = (int64_t)P.m * G;
-    column_fill_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P.rowptr, P.colidx, P.m, P.n, P.colptr,
-                                                                             pl->cursor, pl->keys, P.err);
+    row_expand_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P.rowptr, P.colidx, P.m, pl->rx_row_b, P.err);
     note_launches(1);
 }
 
@@ -145,31 +153,34 @@ int group_width(int64_t nnz, int64_t m) {
     return avg <= 4 ? 4 : avg <= 8 ? 8 : avg <= 16 ? 16 : 32;
 }
 
-template <typename V, int R, int G>
-void launch_colsort_group(spsyrk_plan_s* pl, int64_t first, int64_t count, cudaStream_t st) {
-    if (count <= 0) return;
-    const int64_t threads = count * G;
-    column_sort_group_kernel<V, R, G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(pl->dev, pl->colperm + first, count, pl->keys);
-    note_launches(1);
-}
-
+// stable radix sort of the nonzeros by column id; the last pass writes the column lists and descriptors
 template <typename V>
-spsyrk_status_t sort_columns(spsyrk_plan_s* pl, const int64_t* cs, cudaStream_t st) {
-    launch_colsort_group<V, 1, 8>(pl, cs[1], cs[2] - cs[1], st);
-    launch_colsort_group<V, 1, 16>(pl, cs[2], cs[3] - cs[2], st);
-    launch_colsort_group<V, 1, 32>(pl, cs[3], cs[4] - cs[3], st);
-    launch_colsort_group<V, 2, 32>(pl, cs[4], cs[5] - cs[4], st);
-    launch_colsort_group<V, 4, 32>(pl, cs[5], cs[6] - cs[5], st);
-    launch_colsort_group<V, 8, 32>(pl, cs[6], cs[7] - cs[6], st);
-    const int64_t big = cs[8] - cs[7];
-    if (big > 0) {
-        const uint32_t cb = pow2_at_least((uint64_t)pl->dev.m, 1024u, COL_CHUNK_BITS_MAX);
-        const size_t smem = (size_t)(cb >> 5) * 2 * sizeof(uint32_t);
-        SPSYRK_CUDA_TRY(cudaFuncSetAttribute(column_sort_cta_kernel<V, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        column_sort_cta_kernel<V, 512><<<(unsigned)big, 512, smem, st>>>(pl->dev, pl->colperm + cs[7], pl->keys, cb);
-        note_launches(1);
+spsyrk_status_t sort_by_column(spsyrk_plan_s* pl, cudaStream_t st) {
+    constexpr int BITS = TRANSPOSE_RADIX_BITS;
+    const PlanDev& P = pl->dev;
+    if (P.nnz == 0) return SPSYRK_OK;
+    const int npass = (bits_for((uint64_t)std::max<int64_t>(P.n - 1, 1)) + BITS - 1) / BITS;
+    const uint32_t* src_key = reinterpret_cast<const uint32_t*>(P.colidx);
+    const uint32_t* src_row = pl->rx_row_b;
+    const uint32_t* src_pos = nullptr;  // position in A: the element's own index in the first pass
+    for (int p = 0; p < npass; ++p) {
+        const bool to_a = (p % 2) == 0;
+        uint32_t* dst_key = to_a ? pl->rx_key_a : pl->rx_key_b;
+        uint32_t* dst_row = to_a ? pl->rx_row_a : pl->rx_row_b;
+        uint32_t* dst_pos = to_a ? pl->rx_pos_a : pl->rx_pos_b;
+        if (p == npass - 1) {
+            EmitTransposeFinal<V> emit{P};
+            SPSYRK_CUDA_TRY((radix_pass<BITS, uint32_t>(src_key, src_row, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
+                                                        pl->partials, emit, st)));
+        } else {
+            EmitArrays<uint32_t> emit{dst_key, dst_row, dst_pos};
+            SPSYRK_CUDA_TRY((radix_pass<BITS, uint32_t>(src_key, src_row, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
+                                                        pl->partials, emit, st)));
+        }
+        src_key = dst_key;
+        src_row = dst_row;
+        src_pos = dst_pos;
     }
-    SPSYRK_CUDA_TRY(cudaGetLastError());
     return SPSYRK_OK;
 }
 
@@ -321,6 +332,7 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     if (!plan || !d_rowptr || (nnz > 0 && (!d_colidx || !d_vals))) return SPSYRK_ERR_INVALID_ARG;
     if (*workspace_bytes < need) return SPSYRK_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(d_workspace) % ALIGN) return SPSYRK_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_colidx) % 16) return SPSYRK_ERR_INVALID_ARG;  // tiles of it are copied 16 bytes at a time
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     spsyrk_plan_s* pl = new (std::nothrow) spsyrk_plan_s();
@@ -342,17 +354,14 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     auto fail = [&](spsyrk_status_t s) { delete pl; return s; };
 #define PLAN_TRY(expr) do { if ((expr) != cudaSuccess) return fail(SPSYRK_ERR_CUDA); } while (0)
     PLAN_TRY(cudaMemsetAsync(P.err, 0, sizeof(uint32_t), st));
-    if (n > 0) {
-        PLAN_TRY(cudaMemsetAsync(pl->colcnt, 0, (size_t)n * sizeof(uint32_t), st));
-        PLAN_TRY(cudaMemsetAsync(pl->cursor, 0, (size_t)n * sizeof(uint32_t), st));
-    }
+    if (n > 0) PLAN_TRY(cudaMemsetAsync(pl->colcnt, 0, (size_t)n * sizeof(uint32_t), st));
     // 1. row pointers must be sane before anything indexes with them
     validate_rowptr_kernel<<<(unsigned)((m + 1 + 255) / 256), 256, 0, st>>>(d_rowptr, m, nnz, P.err);
     note_launches(1);
     PLAN_TRY(cudaGetLastError());
     spsyrk_status_t s = read_err(pl, st);
     if (s != SPSYRK_OK) return fail(s);
-    // 2. transpose: histogram, scan, keyed scatter, per-column sort
+    // 2. transpose: column histogram and scan give colptr; explicit row ids; stable radix sort by column
     if (nnz > 0) {
         const unsigned hb = (unsigned)std::min<int64_t>((nnz + 255) / 256, 148 * 32);
         column_histogram_kernel<<<hb, 256, 0, st>>>(d_colidx, nnz, P.n, pl->colcnt, P.err);
@@ -361,22 +370,15 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     PLAN_TRY(exclusive_scan_i64<uint32_t>(pl->colcnt, n, P.colptr, pl->partials, st));
     if (nnz > 0) {
         switch (group_width(nnz, m)) {
-            case 4: launch_fill<4>(pl, st); break;
-            case 8: launch_fill<8>(pl, st); break;
-            case 16: launch_fill<16>(pl, st); break;
-            default: launch_fill<32>(pl, st); break;
+            case 4: launch_row_expand<4>(pl, st); break;
+            case 8: launch_row_expand<8>(pl, st); break;
+            case 16: launch_row_expand<16>(pl, st); break;
+            default: launch_row_expand<32>(pl, st); break;
         }
     }
-    if (n > 0) {
-        column_class_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(P.colptr, P.n, pl->cls);
-        note_launches(1);
-    }
-    PLAN_TRY(bin_items(pl->cls, n, pl->colperm, pl->class_start_dev, pl->blockhist, pl->offsets, pl->partials, st));
-    int64_t cs[NCLASS + 1];
-    PLAN_TRY(cudaMemcpyAsync(cs, pl->class_start_dev, sizeof(cs), cudaMemcpyDeviceToHost, st));
     s = read_err(pl, st);  // synchronises; column ids are known to be in range and rows sorted from here on
     if (s != SPSYRK_OK) return fail(s);
-    s = sv == 8 ? sort_columns<uint64_t>(pl, cs, st) : sort_columns<uint32_t>(pl, cs, st);
+    s = sv == 8 ? sort_by_column<uint64_t>(pl, st) : sort_by_column<uint32_t>(pl, st);
     if (s != SPSYRK_OK) return fail(s);
     // 3. work estimate and row binning
     s = estimate_and_bin(pl, st);

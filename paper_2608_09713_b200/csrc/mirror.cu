@@ -217,6 +217,7 @@ extern "C" spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_
     }
     // step 3: fill
     if (!d_f_vals || (nnz_l > 0 && !d_l_vals)) return SPSYRK_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_l_vals) % 16) return SPSYRK_ERR_INVALID_ARG;  // tiles of it are copied 16 bytes at a time
     if (m == 0) return SPSYRK_OK;
     switch (dtype) {
         case SPSYRK_F64: return mirror_fill<uint64_t>(w, m, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_f_rowptr, d_f_colidx, d_f_vals, st);

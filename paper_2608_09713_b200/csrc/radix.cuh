@@ -80,7 +80,8 @@ struct RadixSmem {
 };
 
 // Emit(dest, key, pa, pb) is called once per element with its position `dest` in the order sorted
-// by the digits seen so far.  pa == nullptr means "payload a is the element's own index".
+// by the digits seen so far.  pa == nullptr (pb == nullptr) means "this payload is the element's own
+// index".
 // All input arrays must be 16-byte aligned.
 template <int BITS, typename PB, typename Emit>
 __global__ void __launch_bounds__(RX_THREADS) radix_scatter_kernel(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pa,
@@ -106,7 +107,7 @@ __global__ void __launch_bounds__(RX_THREADS) radix_scatter_kernel(const uint32_
     rx_tile_load(s_key, keys, tile_base, tile_n);
     rx_cp_async_commit();
     if (pa) rx_tile_load(s_pa, pa, tile_base, tile_n);
-    rx_tile_load(s_pb, pb, tile_base, tile_n);
+    if (pb) rx_tile_load(s_pb, pb, tile_base, tile_n);
     rx_cp_async_commit();
     for (int d = tid; d < RX_WARPS * NB; d += RX_THREADS) wcount[d] = 0;
     rx_cp_async_wait<1>();
@@ -177,7 +178,8 @@ __global__ void __launch_bounds__(RX_THREADS) radix_scatter_kernel(const uint32_
     __syncthreads();
     for (int q = tid; q < tile_n; q += RX_THREADS) {
         const uint32_t d = s_dig[q], src = s_src[q];
-        emit(goff[d] + (int64_t)(q - bin_start[d]), s_key[src], pa ? s_pa[src] : (uint32_t)(tile_base + src), s_pb[src]);
+        emit(goff[d] + (int64_t)(q - bin_start[d]), s_key[src], pa ? s_pa[src] : (uint32_t)(tile_base + src),
+             pb ? s_pb[src] : (PB)(tile_base + src));
     }
 }
 
