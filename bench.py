@@ -166,11 +166,15 @@ def run_ours(args):
     a = W.config(args.workload)
     if args.er_log2m:
         a = W.erdos_renyi(1 << args.er_log2m, 1 << args.er_log2m, 16, W.SEED + 5, np.float64, -1.0, 1.0)
+    if args.zipf_rows:
+        a = W.zipf_binary(args.zipf_rows, 1 << 22, 100, 1.1, W.SEED + 2)
+    if args.rmat_scale:
+        a = W.rmat(args.rmat_scale, 16, W.SEED + 3)
     sv = a.vals.dtype.itemsize
     dname = {np.dtype(np.float64): "f64", np.dtype(np.float32): "f32", np.dtype(np.int32): "i32"}[a.vals.dtype]
     d_rowptr, d_colidx, d_vals = (torch.from_numpy(x).cuda() for x in (a.rowptr, a.colidx, a.vals))
     is_int = a.vals.dtype == np.int32
-    do_mirror = not (args.no_mirror or args.workload == 2)  # the 1e5 x 1e5 dense mirror of config 2 is not asked for
+    do_mirror = not (args.no_mirror or is_int)  # the 1e5 x 1e5 dense mirror of config 2 is not asked for
     stream = torch.cuda.current_stream()
 
     def ev():
@@ -371,6 +375,9 @@ def main():
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--skip-extras", action="store_true", help="timed steps only (for profiler runs)")
+    ap.add_argument("--zipf-rows", type=int, default=0,
+                    help="profiling aid: replace the workload by the binary Zipf recipe with this many rows")
+    ap.add_argument("--rmat-scale", type=int, default=0, help="profiling aid: R-MAT recipe at this scale")
     ap.add_argument("--er-log2m", type=int, default=0,
                     help="profiling aid: replace the workload by the large Erdos-Renyi recipe at m = n = 2**k")
     args = ap.parse_args()

@@ -22,7 +22,7 @@ template <typename V, int THREADS, bool NUMERIC>
 struct CtaRowSmem {
     using Acc = typename AccOf<V>::type;
     static size_t bytes(uint32_t chunk_bits, uint32_t acc_slots) {
-        size_t words = (size_t)(chunk_bits >> 5) * (NUMERIC ? 2 : 1) + 2 * THREADS + 1;
+        size_t words = (size_t)(chunk_bits >> 5) * (NUMERIC ? 2 : 1) + 4 * THREADS + 1;
         words = (words + 3) & ~size_t(3);
         size_t b = words * 4;
         if (NUMERIC) b += (size_t)THREADS * sizeof(Acc) + (size_t)acc_slots * sizeof(Acc);
@@ -40,33 +40,66 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ uint32_t scratch[33];
     __shared__ uint32_t s_sel[2];
+    __shared__ uint32_t s_nlong;
     const uint32_t cw = chunk_bits >> 5;
     uint32_t* bits = reinterpret_cast<uint32_t*>(smem_raw);
     uint32_t* rank = bits + cw;  // numeric only
     uint32_t* loff = bits + (size_t)cw * (NUMERIC ? 2 : 1);
     uint32_t* lstart = loff + THREADS + 1;
-    size_t words = (size_t)cw * (NUMERIC ? 2 : 1) + 2 * THREADS + 1;
+    uint32_t* llen = lstart + THREADS;      // lengths of the batch's lists
+    uint32_t* long_idx = llen + THREADS;    // batch indices of the long lists
+    size_t words = (size_t)cw * (NUMERIC ? 2 : 1) + 4 * THREADS + 1;
     words = (words + 3) & ~size_t(3);
     Acc* la = reinterpret_cast<Acc*>(smem_raw + words * 4);
     Acc* acc = la + THREADS;
 
     const int tid = threadIdx.x;
-    const int32_t rloc = rows[blockIdx.x];
+    // later rows carry longer column prefixes: hand them out first so that the tail of the launch is light
+    const int32_t rloc = rows[gridDim.x - 1 - blockIdx.x];
     const int64_t i = (int64_t)P.r0 + rloc;
     const uint32_t U = P.mode == SPSYRK_TRIL ? (uint32_t)i + 1u : (uint32_t)P.m;
     const int64_t p0 = P.rowptr[i];
     const uint32_t deg = (uint32_t)(P.rowptr[i + 1] - p0);
     const int64_t out_base = NUMERIC ? c_rowptr[rloc] : 0;
-    const uint32_t per = (cw + THREADS - 1) / THREADS;
-    const uint32_t w0 = tid * per;
     uint32_t total_cnt = 0;
 
+    // A row whose range fits one chunk and that holds a column present in every candidate row
+    // (a list as long as the range) is dense: every j occurs, slot = j, no bitmap is needed.
+    bool dense = false;
+    if (U <= chunk_bits) {
+        int hit = 0;
+        for (uint32_t b0 = tid; b0 < deg; b0 += THREADS) hit |= (P.desc[p0 + b0].y == U);
+        dense = __syncthreads_or(hit) != 0;
+    }
+    if (dense && !NUMERIC) {
+        if (tid == 0) cnt[rloc] = (int32_t)U;
+        return;
+    }
+
+    // One partial product: set its bit, or add it into its slot.
+    auto apply = [&](auto what, auto dense_tag, uint32_t rel, Acc a, Acc v, uint32_t s0) {
+        constexpr int WHAT = decltype(what)::value;
+        constexpr bool DENSE = decltype(dense_tag)::value;
+        if (WHAT == CTA_SETBITS) {
+            atomicOr(&bits[rel >> 5], 1u << (rel & 31));
+        } else {
+            const uint32_t slot = (DENSE ? rel : rank[rel >> 5] + __popc(bits[rel >> 5] & ((1u << (rel & 31)) - 1u))) - s0;
+            atomicAdd(&acc[slot], acc_mul(a, v));
+        }
+    };
+
     // Visit every partial product whose j lies in [lo, hi); `whole` skips the per-list search.
-    auto for_each_product = [&](auto what, uint32_t lo, uint32_t hi, bool whole, uint32_t c0, uint32_t s0) {
+    // Lists of at least LONG_LIST entries are walked one after the other by the whole CTA (a lean
+    // loop: two loads and one shared-memory atomic per product); the shorter ones are flattened
+    // through a prefix sum of their lengths so that no lane idles on a short list.
+    constexpr uint32_t LONG_LIST = THREADS / 2;
+    constexpr int UNR = 4;
+    auto for_each_product = [&](auto what, auto dense_tag, uint32_t lo, uint32_t hi, bool whole, uint32_t c0, uint32_t s0) {
         constexpr int WHAT = decltype(what)::value;
         for (uint32_t b0 = 0; b0 < deg; b0 += THREADS) {
             uint32_t sublen = 0, substart = 0;
             Acc a = Acc(0);
+            if (tid == 0) s_nlong = 0;
             if (b0 + tid < deg) {
                 const uint2 d = P.desc[p0 + b0 + tid];
                 if (whole) {
@@ -81,58 +114,129 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                 }
                 if (WHAT == CTA_ACCUM) a = (Acc) static_cast<const V*>(P.vals)[p0 + b0 + tid];
             }
+            const bool is_long = sublen >= LONG_LIST;
             uint32_t T;
-            const uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(sublen, scratch, &T);
+            const uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(is_long ? 0u : sublen, scratch, &T);
             loff[tid] = ex;
             lstart[tid] = substart;
+            llen[tid] = sublen;
             if (WHAT == CTA_ACCUM) la[tid] = a;
             if (tid == 0) loff[THREADS] = T;
+            if (is_long) long_idx[atomicAdd(&s_nlong, 1u)] = tid;
             __syncthreads();
-            uint32_t cur = 0;
-            for (uint32_t item = tid; item < T; item += THREADS) {
-                while (item >= loff[cur + 1]) ++cur;
-                const uint32_t q = lstart[cur] + (item - loff[cur]);
-                const uint32_t rel = (uint32_t)P.at_row[q] - c0;
-                if (WHAT == CTA_SETBITS) {
-                    atomicOr(&bits[rel >> 5], 1u << (rel & 31));
-                } else {
-                    const uint32_t slot = rank[rel >> 5] + __popc(bits[rel >> 5] & ((1u << (rel & 31)) - 1u)) - s0;
-                    atomicAdd(&acc[slot], acc_mul(la[cur], (Acc) static_cast<const V*>(P.at_val)[q]));
+            // short lists, flattened; the current list's bounds, start and factor stay in registers
+            {
+                uint32_t cur = 0, cur_off = 0, next_off = loff[1], cur_start = lstart[0];
+                Acc cur_a = WHAT == CTA_ACCUM ? la[0] : Acc(0);
+                for (uint32_t item0 = tid; item0 < T; item0 += THREADS * UNR) {
+                    uint32_t q[UNR];
+                    Acc av[UNR];
+#pragma unroll
+                    for (int u = 0; u < UNR; ++u) {
+                        const uint32_t item = item0 + u * THREADS;
+                        q[u] = 0xffffffffu;
+                        if (item < T) {
+                            if (item >= next_off) {
+                                do { ++cur; } while (item >= loff[cur + 1]);
+                                cur_off = loff[cur];
+                                next_off = loff[cur + 1];
+                                cur_start = lstart[cur];
+                                if (WHAT == CTA_ACCUM) cur_a = la[cur];
+                            }
+                            q[u] = cur_start + (item - cur_off);
+                            av[u] = cur_a;
+                        }
+                    }
+                    uint32_t rel[UNR];
+                    Acc val[UNR];
+#pragma unroll
+                    for (int u = 0; u < UNR; ++u) {
+                        rel[u] = 0;
+                        val[u] = Acc(0);
+                        if (q[u] != 0xffffffffu) {
+                            rel[u] = (uint32_t)P.at_row[q[u]] - c0;
+                            if (WHAT == CTA_ACCUM) val[u] = (Acc) static_cast<const V*>(P.at_val)[q[u]];
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < UNR; ++u)
+                        if (q[u] != 0xffffffffu) apply(what, dense_tag, rel[u], av[u], val[u], s0);
                 }
+            }
+            // long lists, one after the other
+            const uint32_t nlong = s_nlong;
+            for (uint32_t li = 0; li < nlong; ++li) {
+                const uint32_t t = long_idx[li];
+                const uint32_t len = llen[t];
+                const int32_t* __restrict__ rowp = P.at_row + lstart[t];
+                const V* __restrict__ valp = static_cast<const V*>(P.at_val) + lstart[t];
+                const Acc fa = WHAT == CTA_ACCUM ? la[t] : Acc(0);
+                uint32_t e = tid;
+                for (; e + (UNR - 1) * THREADS < len; e += UNR * THREADS) {
+                    uint32_t rel[UNR];
+                    Acc val[UNR];
+#pragma unroll
+                    for (int u = 0; u < UNR; ++u) {
+                        rel[u] = (uint32_t)rowp[e + u * THREADS] - c0;
+                        val[u] = WHAT == CTA_ACCUM ? (Acc)valp[e + u * THREADS] : Acc(0);
+                    }
+#pragma unroll
+                    for (int u = 0; u < UNR; ++u) apply(what, dense_tag, rel[u], fa, val[u], s0);
+                }
+                for (; e < len; e += THREADS)
+                    apply(what, dense_tag, (uint32_t)rowp[e] - c0, fa, WHAT == CTA_ACCUM ? (Acc)valp[e] : Acc(0), s0);
             }
             __syncthreads();
         }
     };
+    const std::integral_constant<int, CTA_SETBITS> SET{};
+    const std::integral_constant<int, CTA_ACCUM> ACC{};
+    const std::true_type IS_DENSE{};
+    const std::false_type NOT_DENSE{};
 
     for (uint32_t c0 = 0; c0 < U; c0 += chunk_bits) {
         const uint32_t c1 = min(c0 + chunk_bits, U);
         const bool single_chunk = (c0 == 0 && c1 == U);
-        for (uint32_t w = tid; w < cw; w += THREADS) bits[w] = 0;
-        __syncthreads();
-        for_each_product(std::integral_constant<int, CTA_SETBITS>{}, c0, c1, single_chunk, c0, 0u);
-        uint32_t s = 0;
-        for (uint32_t w = w0; w < w0 + per && w < cw; ++w) s += __popc(bits[w]);
-        uint32_t tot;
-        uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(s, scratch, &tot);
-        if (NUMERIC) {
-            for (uint32_t w = w0; w < w0 + per && w < cw; ++w) { rank[w] = ex; ex += __popc(bits[w]); }
+        const uint32_t cwa = (c1 - c0 + 31) >> 5;  // words of the bitmap this chunk uses
+        const uint32_t per = (cwa + THREADS - 1) / THREADS;
+        const uint32_t w0 = tid * per;
+        uint32_t tot = c1 - c0;
+        if (!dense) {
+            for (uint32_t w = tid; w < cwa; w += THREADS) bits[w] = 0;
             __syncthreads();
+            for_each_product(SET, NOT_DENSE, c0, c1, single_chunk, c0, 0u);
+            uint32_t s = 0;
+            for (uint32_t w = w0; w < w0 + per && w < cwa; ++w) s += __popc(bits[w]);
+            uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(s, scratch, &tot);
+            if (NUMERIC) {
+                for (uint32_t w = w0; w < w0 + per && w < cwa; ++w) { rank[w] = ex; ex += __popc(bits[w]); }
+                __syncthreads();
+            }
+        }
+        if (NUMERIC) {
             const int64_t ob = out_base + total_cnt;
-            // column ids straight from the bitmap
-            for (uint32_t w = tid; w < cw; w += THREADS) {
-                uint32_t b = bits[w], r = rank[w];
-                while (b) {
-                    const int bit = __ffs(b) - 1;
-                    c_colidx[ob + r] = (int32_t)(c0 + (w << 5) + bit);
-                    ++r;
-                    b &= b - 1;
+            if (dense) {
+                for (uint32_t t = tid; t < tot; t += THREADS) c_colidx[ob + t] = (int32_t)(c0 + t);
+            } else {
+                // column ids straight from the bitmap
+                for (uint32_t w = tid; w < cwa; w += THREADS) {
+                    uint32_t b = bits[w], r = rank[w];
+                    while (b) {
+                        const int bit = __ffs(b) - 1;
+                        c_colidx[ob + r] = (int32_t)(c0 + (w << 5) + bit);
+                        ++r;
+                        b &= b - 1;
+                    }
                 }
             }
             for (uint32_t s0 = 0; s0 < tot; s0 += acc_slots) {
                 const uint32_t s1 = min(s0 + acc_slots, tot);
                 const bool single_tile = (s0 == 0 && s1 == tot);
                 uint32_t jlo = c0, jhi = c1;
-                if (!single_tile) {
+                if (!single_tile && dense) {
+                    jlo = c0 + s0;
+                    jhi = c0 + s1;
+                } else if (!single_tile) {
                     if (tid < 2) {
                         const uint32_t sl = tid == 0 ? s0 : s1;
                         uint32_t res;
@@ -140,7 +244,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                         else if (tid == 1 && s1 == tot) res = c1;
                         else {
                             // last word whose rank is <= sl holds slot sl
-                            uint32_t lo_w = 0, hi_w = cw;
+                            uint32_t lo_w = 0, hi_w = cwa;
                             while (hi_w - lo_w > 1) {
                                 uint32_t mid = (lo_w + hi_w) >> 1;
                                 if (rank[mid] <= sl) lo_w = mid; else hi_w = mid;
@@ -157,7 +261,8 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                 }
                 for (uint32_t t = tid; t < s1 - s0; t += THREADS) acc[t] = Acc(0);
                 __syncthreads();
-                for_each_product(std::integral_constant<int, CTA_ACCUM>{}, jlo, jhi, single_chunk && single_tile, c0, s0);
+                if (dense) for_each_product(ACC, IS_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0);
+                else for_each_product(ACC, NOT_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0);
                 for (uint32_t t = tid; t < s1 - s0; t += THREADS) c_vals[ob + s0 + t] = (V)acc[t];
                 __syncthreads();
             }
