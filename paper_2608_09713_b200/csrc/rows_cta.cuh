@@ -124,43 +124,54 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
             if (tid == 0) loff[THREADS] = T;
             if (is_long) long_idx[atomicAdd(&s_nlong, 1u)] = tid;
             __syncthreads();
-            // short lists, flattened; the current list's bounds, start and factor stay in registers
+            // short lists, flattened: every thread takes a contiguous run of items (so that moving
+            // from one list to the next is a step, not a search), UNR loads in flight at a time
             {
-                uint32_t cur = 0, cur_off = 0, next_off = loff[1], cur_start = lstart[0];
-                Acc cur_a = WHAT == CTA_ACCUM ? la[0] : Acc(0);
-                for (uint32_t item0 = tid; item0 < T; item0 += THREADS * UNR) {
-                    uint32_t q[UNR];
-                    Acc av[UNR];
+                const uint32_t ipt = (T + THREADS - 1) / THREADS;
+                const uint32_t first = min((uint32_t)tid * ipt, T), last = min(first + ipt, T);
+                if (first < last) {
+                    uint32_t lo_l = 0, hi_l = THREADS;  // last list whose offset is <= first
+                    while (hi_l - lo_l > 1) {
+                        const uint32_t mid = (lo_l + hi_l) >> 1;
+                        if (loff[mid] <= first) lo_l = mid; else hi_l = mid;
+                    }
+                    uint32_t cur = lo_l, cur_off = loff[cur], next_off = loff[cur + 1], cur_start = lstart[cur];
+                    Acc cur_a = WHAT == CTA_ACCUM ? la[cur] : Acc(0);
+                    for (uint32_t item0 = first; item0 < last; item0 += UNR) {
+                        uint32_t q[UNR];
+                        Acc av[UNR];
 #pragma unroll
-                    for (int u = 0; u < UNR; ++u) {
-                        const uint32_t item = item0 + u * THREADS;
-                        q[u] = 0xffffffffu;
-                        if (item < T) {
-                            if (item >= next_off) {
-                                do { ++cur; } while (item >= loff[cur + 1]);
-                                cur_off = loff[cur];
-                                next_off = loff[cur + 1];
-                                cur_start = lstart[cur];
-                                if (WHAT == CTA_ACCUM) cur_a = la[cur];
+                        for (int u = 0; u < UNR; ++u) {
+                            const uint32_t item = item0 + u;
+                            q[u] = 0xffffffffu;
+                            av[u] = Acc(0);
+                            if (item < last) {
+                                if (item >= next_off) {
+                                    do { ++cur; } while (item >= loff[cur + 1]);
+                                    cur_off = loff[cur];
+                                    next_off = loff[cur + 1];
+                                    cur_start = lstart[cur];
+                                    if (WHAT == CTA_ACCUM) cur_a = la[cur];
+                                }
+                                q[u] = cur_start + (item - cur_off);
+                                av[u] = cur_a;
                             }
-                            q[u] = cur_start + (item - cur_off);
-                            av[u] = cur_a;
                         }
-                    }
-                    uint32_t rel[UNR];
-                    Acc val[UNR];
+                        uint32_t rel[UNR];
+                        Acc val[UNR];
 #pragma unroll
-                    for (int u = 0; u < UNR; ++u) {
-                        rel[u] = 0;
-                        val[u] = Acc(0);
-                        if (q[u] != 0xffffffffu) {
-                            rel[u] = (uint32_t)P.at_row[q[u]] - c0;
-                            if (WHAT == CTA_ACCUM) val[u] = (Acc) static_cast<const V*>(P.at_val)[q[u]];
+                        for (int u = 0; u < UNR; ++u) {
+                            rel[u] = 0;
+                            val[u] = Acc(0);
+                            if (q[u] != 0xffffffffu) {
+                                rel[u] = (uint32_t)P.at_row[q[u]] - c0;
+                                if (WHAT == CTA_ACCUM) val[u] = (Acc) static_cast<const V*>(P.at_val)[q[u]];
+                            }
                         }
-                    }
 #pragma unroll
-                    for (int u = 0; u < UNR; ++u)
-                        if (q[u] != 0xffffffffu) apply(what, dense_tag, rel[u], av[u], val[u], s0);
+                        for (int u = 0; u < UNR; ++u)
+                            if (q[u] != 0xffffffffu) apply(what, dense_tag, rel[u], av[u], val[u], s0);
+                    }
                 }
             }
             // long lists, one after the other
