@@ -97,8 +97,7 @@ __global__ void __launch_bounds__(RX_THREADS) radix_scatter_kernel(const uint32_
     uint32_t* s_pa = s_key + RX_TILE;                                  // [TILE] source order
     uint32_t* wcount = s_pa + RX_TILE;                                 // [WARPS][NB]
     uint32_t* bin_start = wcount + RX_WARPS * NB;                      // [NB]
-    uint16_t* s_src = reinterpret_cast<uint16_t*>(bin_start + NB);     // [TILE] source index of the element at sorted slot q
-    uint16_t* s_dig = s_src + RX_TILE;                                 // [TILE] its digit
+    uint32_t* s_perm = bin_start + NB;                                 // [TILE] (digit << 16) | source index of sorted slot q
 
     const int tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
     const int64_t tile_base = (int64_t)blockIdx.x * RX_TILE;
@@ -170,16 +169,18 @@ __global__ void __launch_bounds__(RX_THREADS) radix_scatter_kernel(const uint32_
         if (!(rk[i] & 0x80000000u)) {
             const uint32_t d = (rk[i] >> 12) & 0xfffu;
             const uint32_t q = bin_start[d] + mycount[d] + (rk[i] & 0xfffu);
-            s_src[q] = (uint16_t)(warp * RX_CHUNK + i * 32 + lane);
-            s_dig[q] = (uint16_t)d;
+            s_perm[q] = (d << 16) | (uint32_t)(warp * RX_CHUNK + i * 32 + lane);
         }
     }
     rx_cp_async_wait<0>();
     __syncthreads();
+    // slot q of digit d goes to goff[d] + (q - bin_start[d]): fold the two tables into one
+    for (int d = tid; d < NB; d += RX_THREADS) goff[d] -= (int64_t)bin_start[d];
+    __syncthreads();
     for (int q = tid; q < tile_n; q += RX_THREADS) {
-        const uint32_t d = s_dig[q], src = s_src[q];
-        emit(goff[d] + (int64_t)(q - bin_start[d]), s_key[src], pa ? s_pa[src] : (uint32_t)(tile_base + src),
-             pb ? s_pb[src] : (PB)(tile_base + src));
+        const uint32_t pd = s_perm[q];
+        const uint32_t src = pd & 0xffffu;
+        emit(goff[pd >> 16] + q, s_key[src], pa ? s_pa[src] : (uint32_t)(tile_base + src), pb ? s_pb[src] : (PB)(tile_base + src));
     }
 }
 
