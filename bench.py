@@ -34,7 +34,7 @@ METRIC = "tril_syrk_useful_multiply_adds_per_s"
 UNIT = "MAC/s"
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (bytes per useful multiply-add, multiplied by the launch's multiply-adds); None = not captured.
-NCU_TRAFFIC_BYTES_PER_MAC = None
+NCU_TRAFFIC_BYTES_PER_MAC = 34.5
 
 
 def measured_peaks():
@@ -87,6 +87,22 @@ class ClockSampler:
                     reasons.add(nm)
         return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
                 "samples": len(mhz)}
+
+
+def max_over_ranks(x: float, device="cpu") -> float:
+    """Maximum of a per-rank number over all ranks (the job is as slow as its slowest replica)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Replicas: every rank processes `units_per_rank` per step; the job's rate counts all of them."""
+    return world * units_per_rank / (ms_per_step / 1e3)
 
 
 def class_of_rows(work, deg):
@@ -248,17 +264,14 @@ def run_ours(args):
     clocks = sampler.stop(t0, t1) if rank == 0 else None
     total_ms = results[0]["marks"][0].elapsed_time(results[-1]["marks"][-1])
     ms_per_step = total_ms / args.steps
-    if world > 1:
-        t = torch.tensor([ms_per_step], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step = float(t.item())
+    ms_per_step = max_over_ranks(ms_per_step, "cuda")
     names = ["plan", "symbolic", "numeric", "mirror", "jaccard"]
     phases = {nm: float(np.mean([r["marks"][i].elapsed_time(r["marks"][i + 1]) for r in results])) for i, nm in enumerate(names)}
     work_total, class_rows = B.spsyrk_plan_stats(results[-1]["plan"])
     nnz_c, nnz_f = results[-1]["nnz"], results[-1]["nnz_full"]
     sym_ms = np.mean([B.spsyrk_plan_timings(r["plan"])[0] for r in results], axis=0)
     num_ms = np.mean([B.spsyrk_plan_timings(r["plan"])[1] for r in results], axis=0)
-    value = world * work_total / (ms_per_step / 1e3)
+    value = whole_job_rate(work_total, world, ms_per_step)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dname,
@@ -266,7 +279,7 @@ def run_ours(args):
             "config": {"workload": a.name, "m": a.m, "n": a.n, "nnz_a": a.nnz, "multiply_adds": work_total, "nnz_c_l": nnz_c,
                        "nnz_full": nnz_f, "step": "plan+symbolic+numeric" + ("+mirror" if do_mirror else "") + ("+jaccard" if is_int else ""),
                        "l2_policy": "inputs_larger_than_l2", "parallelism": f"replicas x{world}"},
-            "nnz_per_s": world * nnz_c / (ms_per_step / 1e3), "phases_ms": phases,
+            "nnz_per_s": whole_job_rate(nnz_c, world, ms_per_step), "phases_ms": phases,
             "numeric_class_ms": [float(x) for x in num_ms], "symbolic_class_ms": [float(x) for x in sym_ms],
             "class_rows": class_rows, "gpu_launches": int(launches), "clocks": clocks}
 
@@ -344,13 +357,10 @@ def run_ours(args):
             B.spsyrk_host_tril(a.m, a.n, *h_in, out=out)
         barrier()
         e2e_ms = (time.perf_counter() - ts) * 1e3 / args.steps
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e2e_ms, "cuda")
         h2d = a.rowptr.nbytes + a.colidx.nbytes + a.vals.nbytes
         d2h = 8 * (a.m + 1) + nnz_c * (4 + sv)
-        line["e2e"] = {"value": world * work_total / (e2e_ms / 1e3), "unit": UNIT, "ms_per_step": e2e_ms,
+        line["e2e"] = {"value": whole_job_rate(work_total, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                        "what": "spsyrk_host_tril: H2D of A, plan+symbolic+numeric, D2H of C_L (mirror not included)"}
 
