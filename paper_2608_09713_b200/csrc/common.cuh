@@ -96,6 +96,17 @@ __device__ __forceinline__ uint32_t kmin<uint32_t>(uint32_t a, uint32_t b) { ret
 template <>
 __device__ __forceinline__ uint32_t kmax<uint32_t>(uint32_t a, uint32_t b) { return max(a, b); }
 
+// x -> ~x for every key when `flip`, else unchanged.  ~x = -x - 1, written as x * c + d with
+// (c, d) = (-1, -1) or (1, 0): an integer multiply-add, which issues on the FMA pipe and leaves the
+// ALU pipe (busy with the min/max of the network) alone.
+template <typename K, int R>
+__device__ __forceinline__ void flip_keys(K (&x)[R], bool flip) {
+    const K c = flip ? ~K(0) : K(1);
+    const K d = flip ? ~K(0) : K(0);
+#pragma unroll
+    for (int r = 0; r < R; ++r) x[r] = x[r] * c + d;
+}
+
 template <typename K, int R, int G = 32>
 __device__ __forceinline__ void group_bitonic_sort(K (&x)[R]) {
     static_assert((R & (R - 1)) == 0 && (G & (G - 1)) == 0 && G <= 32, "powers of two");
@@ -106,14 +117,10 @@ __device__ __forceinline__ void group_bitonic_sort(K (&x)[R]) {
         if (k >= R && k < G * R) {
             // direction of this level is per lane: descending lanes work on complemented keys
             const bool want = (gl & (k / R)) != 0;
-            const K m = (want != flipped) ? ~K(0) : K(0);
-#pragma unroll
-            for (int r = 0; r < R; ++r) x[r] ^= m;
+            flip_keys<K, R>(x, want != flipped);
             flipped = want;
         } else if (k == G * R && G * R > R) {
-            const K m = flipped ? ~K(0) : K(0);
-#pragma unroll
-            for (int r = 0; r < R; ++r) x[r] ^= m;
+            flip_keys<K, R>(x, flipped);
             flipped = false;
         }
 #pragma unroll

@@ -114,3 +114,36 @@ def test_full_size_configuration(B, idx):
             lo, hi = int(rp_h[r]), int(rp_h[r + 1])
             assert torch.equal(f_colidx[int(frp[r]):int(frp[r]) + hi - lo], ci[lo:hi])
             assert torch.equal(f_vals[int(frp[r]):int(frp[r]) + hi - lo], cv[lo:hi])
+
+
+def test_more_than_2_pow_22_rows_uses_wide_sort_keys(B):
+    """Above 2^22 rows the warp-class sort keys no longer fit 32 bits; the 64-bit variant runs."""
+    m = (1 << 22) + 12345
+    a = W.erdos_renyi(m, 300_000, 3, 4242, np.float64, -1.0, 1.0)
+    d = (torch.from_numpy(a.rowptr).cuda(), torch.from_numpy(a.colidx).cuda(), torch.from_numpy(a.vals).cuda())
+    rp, ci, cv, plan = B.tril_syrk(a.m, a.n, *d)
+    torch.cuda.synchronize()
+    rp_h = rp.cpu().numpy()
+    dk = np.bincount(a.colidx, minlength=a.n).astype(np.int64)
+    assert B.spsyrk_plan_stats(plan)[0] == int((dk * (dk + 1) // 2).sum())
+    cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
+    rows = sample_rows(a.m, np.diff(a.rowptr), 60, 9)
+    check_rows_against_oracle(a, cols, oracle.TRIL, rows, rp_h, ci, cv)
+    f_rowptr, f_colidx, f_vals = B.spsyrk_mirror(a.m, rp, ci, cv)
+    check_rows_against_oracle(a, cols, oracle.FULL, rows[:30], f_rowptr.cpu().numpy(), f_colidx, f_vals)
+
+
+def test_row_tiles_at_scale(B):
+    """Configuration 5's recipe at 2^19 rows in five ragged row tiles equals the untiled result bit for bit."""
+    a = W.erdos_renyi(1 << 19, 1 << 19, 16, W.SEED + 5, np.float64, -1.0, 1.0)
+    d = (torch.from_numpy(a.rowptr).cuda(), torch.from_numpy(a.colidx).cuda(), torch.from_numpy(a.vals).cuda())
+    rp, ci, cv, plan = B.tril_syrk(a.m, a.n, *d)
+    cuts = [0, 100_001, 100_002, 262_144, 500_000, a.m]
+    cols, vals, counts = [], [], []
+    for r0, r1 in zip(cuts[:-1], cuts[1:]):
+        B.spsyrk_plan_set_rows(plan, r0, r1)
+        trp, tci, tcv, _ = B.tril_syrk(a.m, a.n, *d, row_begin=r0, row_end=r1, plan=plan)
+        cols.append(tci); vals.append(tcv); counts.append(trp[1:] - trp[:-1])
+    assert torch.equal(torch.cat(counts), rp[1:] - rp[:-1])
+    assert torch.equal(torch.cat(cols), ci)
+    assert torch.equal(torch.cat(vals), cv)

@@ -239,3 +239,41 @@ def test_host_entry_point(B):
     ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL)
     assert np.array_equal(rp.numpy(), ref.rowptr) and np.array_equal(ci.numpy(), ref.colidx)
     check_values(cv.numpy(), ref, a.vals.dtype)
+
+
+# ------------------------------------------------------------------ further dtypes and error paths
+def test_int32_general_values_and_fp32_light_rows(B):
+    rng = np.random.default_rng(11)
+    a = W.erdos_renyi(3000, 2500, 9, 123, np.float64, 0.0, 1.0)
+    ai = W.CSR(a.m, a.n, a.rowptr, a.colidx, rng.integers(-50, 51, size=a.nnz).astype(np.int32))
+    run_and_compare(B, ai, 0)
+    run_and_compare(B, ai, 1)
+    af = W.CSR(a.m, a.n, a.rowptr, a.colidx, (rng.random(a.nnz) * 2 - 1).astype(np.float32))
+    run_and_compare(B, af, 0)
+    hf = W.hypergraph(20_000, 5_000, 77)
+    run_and_compare(B, W.CSR(hf.m, hf.n, hf.rowptr, hf.colidx, hf.vals.astype(np.float32)), 0)
+
+
+def test_workspace_and_alignment_errors(B):
+    import ctypes
+    a = W.small(1)
+    rowptr, colidx, vals = dev(a)
+    need = B.spsyrk_plan_workspace_bytes(a.m, a.n, a.nnz, torch.float64)
+    small_ws = torch.empty(need // 2, dtype=torch.uint8, device="cuda")
+    with pytest.raises(AssertionError):
+        B.spsyrk_plan(a.m, a.n, rowptr, colidx, vals, workspace=small_ws)
+    sz = ctypes.c_size_t(small_ws.numel())
+    h = ctypes.c_void_p()
+    st = B._lib.spsyrk_plan(ctypes.byref(h), a.m, a.n, a.nnz, B._p(rowptr), B._p(colidx), B._p(vals), 0, 0, 0, a.m,
+                            B._p(small_ws), ctypes.byref(sz), None)
+    assert st == 3                                                      # workspace too small
+    ws = torch.empty(need + 64, dtype=torch.uint8, device="cuda")
+    sz = ctypes.c_size_t(need)
+    st = B._lib.spsyrk_plan(ctypes.byref(h), a.m, a.n, a.nnz, B._p(rowptr), B._p(colidx), B._p(vals), 0, 0, 0, a.m,
+                            ctypes.c_void_p(ws.data_ptr() + 8), ctypes.byref(sz), None)
+    assert st == 1                                                      # misaligned workspace
+    shifted = torch.empty(a.nnz + 1, dtype=torch.int32, device="cuda")
+    shifted[1:] = colidx
+    st = B._lib.spsyrk_plan(ctypes.byref(h), a.m, a.n, a.nnz, B._p(rowptr), ctypes.c_void_p(shifted.data_ptr() + 4),
+                            B._p(vals), 0, 0, 0, a.m, B._p(ws), ctypes.byref(sz), None)
+    assert st == 1                                                      # column ids not 16-byte aligned
