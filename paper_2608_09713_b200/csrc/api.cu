@@ -215,8 +215,13 @@ template <int N>
 void launch_symbolic_warp(spsyrk_plan_s* pl, int c, cudaStream_t st) {
     const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
     if (count <= 0) return;
-    symbolic_warp_kernel<N><<<(unsigned)((count + ROW_WARPS - 1) / ROW_WARPS), ROW_WARPS * 32, 0, st>>>(
-        pl->dev, pl->perm + pl->class_start[c], count, pl->cnt);
+    constexpr int SW = symbolic_warps(N);
+    auto kern = symbolic_warp_kernel<N>;
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, SW * 32, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const int64_t want = (count + SW - 1) / SW;
+    const int64_t cap = (int64_t)pl->sm_count * per_sm;
+    kern<<<(unsigned)std::min(want, cap), SW * 32, 0, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, pl->cnt);
     note_launches(1);
 }
 

@@ -14,59 +14,12 @@
 
 namespace spsyrk {
 
-constexpr int ROW_WARPS = 8;  // warps (rows) per CTA in the symbolic warp-class kernel
+// warps per CTA of the symbolic warp-class kernel (static shared memory stays under 48 KB)
+__host__ __device__ constexpr int symbolic_warps(int n) { return n >= 512 ? 4 : 8; }
 // warps per CTA of the numeric warp-class kernel: keeps static shared memory under 48 KB
 __host__ __device__ constexpr int numeric_warps(int n) { return n >= 512 ? 2 : n >= 256 ? 4 : 8; }
 // register budget: at least this many CTAs of the numeric kernel must fit on an SM
 __host__ __device__ constexpr int numeric_min_ctas(int n) { return n == 256 ? 6 : 1; }
-
-template <int N>
-__global__ void __launch_bounds__(ROW_WARPS * 32) symbolic_warp_kernel(PlanDev P, const int32_t* __restrict__ rows, int64_t nrows,
-                                                                       int32_t* __restrict__ cnt) {
-    constexpr int T = 2 * N;  // hash slots per warp
-    constexpr int RND = N / 32;
-    constexpr int SHIFT = 32 - ilog2_ce(T);
-    __shared__ uint32_t s_tab[ROW_WARPS][T];
-    __shared__ uint32_t s_off[ROW_WARPS][32];
-    const int warp = threadIdx.x >> 5, lane = lane_id();
-    const int64_t widx = (int64_t)blockIdx.x * ROW_WARPS + warp;
-    if (widx >= nrows) return;
-    const int32_t rloc = rows[widx];
-    const int64_t i = (int64_t)P.r0 + rloc;
-    const int64_t p0 = P.rowptr[i];
-    const int deg = (int)(P.rowptr[i + 1] - p0);
-    uint2 d = lane < deg ? P.desc[p0 + lane] : make_uint2(0u, 0u);
-    const uint32_t incl = warp_inclusive_scan(d.y);
-    const uint32_t w = __shfl_sync(FULL_MASK, incl, 31);
-    s_off[warp][lane] = lane < deg ? incl - d.y : 0xffffffffu;
-#pragma unroll
-    for (int s = lane; s < T; s += 32) s_tab[warp][s] = 0xffffffffu;
-    __syncwarp();
-    int local = 0;
-#pragma unroll
-    for (int r = 0; r < RND; ++r) {
-        if ((uint32_t)(r * 32) < w) {  // warp-uniform
-            const uint32_t t = r * 32 + lane;
-            int s = 0;
-#pragma unroll
-            for (int st = 16; st > 0; st >>= 1)
-                if (s_off[warp][s + st] <= t) s += st;
-            const uint32_t start = __shfl_sync(FULL_MASK, d.x, s);
-            if (t < w) {
-                const uint32_t j = (uint32_t)P.at_row[start + (t - s_off[warp][s])];
-                uint32_t h = (j * 2654435761u) >> SHIFT;
-                for (int probe = 0; probe < T; ++probe) {  // bounded: the table is at most half full
-                    uint32_t old = atomicCAS(&s_tab[warp][h], 0xffffffffu, j);
-                    if (old == 0xffffffffu) { ++local; break; }
-                    if (old == j) break;
-                    h = (h + 1) & (T - 1);
-                }
-            }
-        }
-    }
-    local = warp_reduce_sum(local);
-    if (lane == 0) cnt[rloc] = local;
-}
 
 // Asynchronous global -> shared copies of 4 or 8 bytes (no register staging), grouped per thread.
 template <int BYTES>
@@ -261,6 +214,86 @@ __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) nu
     }
     cp_async_wait<0>();
     (void)rloc_n;
+}
+
+// Symbolic pass for light rows: the same persistent, software-pipelined walk as the numeric kernel
+// (header, descriptors and column-list row ids of later rows in flight while a row is counted), but
+// only the row ids are gathered and they go into a per-warp hash set; the count is the number of
+// successful inserts.
+template <int N>
+__global__ void __launch_bounds__(symbolic_warps(N) * 32) symbolic_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows,
+                                                                       int32_t* __restrict__ cnt) {
+    constexpr int SW = symbolic_warps(N);
+    constexpr int T = 2 * N;  // hash slots per warp
+    constexpr int R = N / 32;
+    constexpr int SHIFT = 32 - ilog2_ce(T);
+    __shared__ uint32_t s_tab[SW][T];
+    __shared__ uint32_t s_j[SW][2][N];
+    const int warp = threadIdx.x >> 5, lane = lane_id();
+    const int64_t stride = (int64_t)gridDim.x * SW;
+    int64_t n = (int64_t)blockIdx.x * SW + warp;
+    if (n >= nrows) return;
+
+    const uint4 none = make_uint4(0u, 0u, 0u, 0u);
+    auto load_hdr = [&](int64_t idx) { return idx < nrows ? hdr[idx] : none; };
+    auto load_desc = [&](const uint4& h) { return (uint32_t)lane < h.z ? P.desc[(int64_t)h.y + lane] : make_uint2(0u, 0u); };
+    auto issue = [&](const uint4& h, const uint2& d, int b) -> uint32_t {
+        const bool live = (uint32_t)lane < h.z;
+        const uint32_t incl = warp_inclusive_scan(d.y);
+        const uint32_t w = __shfl_sync(FULL_MASK, incl, 31);
+        const uint32_t off = live ? incl - d.y : 0xffffffffu;
+        const uint32_t smo = d.x - off;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if ((uint32_t)(r * 32) < w) {  // warp-uniform
+                const uint32_t rel = off - (uint32_t)(r * 32);
+                const uint32_t before = __popc(__ballot_sync(FULL_MASK, off <= (uint32_t)(r * 32)));
+                const uint32_t startbits = __reduce_or_sync(FULL_MASK, (rel - 1u < 31u) ? (1u << rel) : 0u);
+                const uint32_t s = before - 1u + __popc(startbits & (0xfffffffeu >> (31 - lane)));
+                const uint32_t q = r * 32 + lane + __shfl_sync(FULL_MASK, smo, s & 31);
+                if ((uint32_t)(r * 32 + lane) < w) cp_async<4>(&s_j[warp][b][r * 32 + lane], P.at_row + q);
+            }
+        }
+        cp_async_commit();
+        return w;
+    };
+
+    uint4 h0 = load_hdr(n), hB = load_hdr(n + stride), hA = load_hdr(n + 2 * stride);
+    uint2 d0 = load_desc(h0);
+    uint2 dB = load_desc(hB);
+    uint32_t rloc_n = h0.x;
+    uint32_t w_n = issue(h0, d0, 0);
+    int b = 0;
+    for (; n < nrows; n += stride, b ^= 1) {
+        const uint4 hNew = load_hdr(n + 3 * stride);
+        const uint2 dNew = load_desc(hA);
+        const uint32_t w_next = issue(hB, dB, b ^ 1);
+#pragma unroll
+        for (int s = lane; s < T; s += 32) s_tab[warp][s] = 0xffffffffu;
+        cp_async_wait<1>();
+        __syncwarp();
+        int local = 0;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const uint32_t t = r * 32 + lane;
+            if (t < w_n) {
+                const uint32_t j = s_j[warp][b][t];
+                uint32_t h = (j * 2654435761u) >> SHIFT;
+                for (int probe = 0; probe < T; ++probe) {  // bounded: the table is at most half full
+                    const uint32_t old = atomicCAS(&s_tab[warp][h], 0xffffffffu, j);
+                    if (old == 0xffffffffu) { ++local; break; }
+                    if (old == j) break;
+                    h = (h + 1) & (T - 1);
+                }
+            }
+        }
+        local = warp_reduce_sum(local);
+        if (lane == 0) cnt[rloc_n] = local;
+        __syncwarp();  // the table and buffer b are reused by the next rows
+        rloc_n = hB.x; w_n = w_next;
+        hB = hA; dB = dNew; hA = hNew;
+    }
+    cp_async_wait<0>();
 }
 
 }  // namespace spsyrk
