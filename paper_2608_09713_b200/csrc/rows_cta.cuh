@@ -22,7 +22,7 @@ template <typename V, int THREADS, bool NUMERIC>
 struct CtaRowSmem {
     using Acc = typename AccOf<V>::type;
     static size_t bytes(uint32_t chunk_bits, uint32_t acc_slots) {
-        size_t words = (size_t)(chunk_bits >> 5) * (NUMERIC ? 2 : 1) + 4 * THREADS + 1;
+        size_t words = (size_t)(chunk_bits >> 5) * (NUMERIC ? 2 : 1) + 5 * THREADS + 1;
         words = (words + 3) & ~size_t(3);
         size_t b = words * 4;
         if (NUMERIC) b += (size_t)THREADS * sizeof(Acc) + (size_t)acc_slots * sizeof(Acc);
@@ -48,7 +48,8 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     uint32_t* lstart = loff + THREADS + 1;
     uint32_t* llen = lstart + THREADS;      // lengths of the batch's lists
     uint32_t* long_idx = llen + THREADS;    // batch indices of the long lists
-    size_t words = (size_t)cw * (NUMERIC ? 2 : 1) + 4 * THREADS + 1;
+    uint32_t* lprev = long_idx + THREADS;   // where the previous slot tile ended inside each list
+    size_t words = (size_t)cw * (NUMERIC ? 2 : 1) + 5 * THREADS + 1;
     words = (words + 3) & ~size_t(3);
     Acc* la = reinterpret_cast<Acc*>(smem_raw + words * 4);
     Acc* acc = la + THREADS;
@@ -94,7 +95,10 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     // through a prefix sum of their lengths so that no lane idles on a short list.
     constexpr uint32_t LONG_LIST = THREADS / 2;
     constexpr int UNR = 4;
-    auto for_each_product = [&](auto what, auto dense_tag, uint32_t lo, uint32_t hi, bool whole, uint32_t c0, uint32_t s0) {
+    // `resume`: the range starts where the previous call's range ended (consecutive slot tiles of a row
+    // with at most THREADS lists), so each list's lower end is remembered instead of searched again.
+    auto for_each_product = [&](auto what, auto dense_tag, uint32_t lo, uint32_t hi, bool whole, uint32_t c0, uint32_t s0,
+                                bool resume) {
         constexpr int WHAT = decltype(what)::value;
         for (uint32_t b0 = 0; b0 < deg; b0 += THREADS) {
             uint32_t sublen = 0, substart = 0;
@@ -107,8 +111,9 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     sublen = d.y;
                 } else {
                     const int32_t* lst = P.at_row + d.x;
-                    const uint32_t a0 = lo == 0 ? 0u : lower_bound_i32(lst, d.y, (int32_t)lo);
-                    const uint32_t a1 = lower_bound_i32(lst, d.y, (int32_t)hi);
+                    const uint32_t a0 = lo == 0 ? 0u : resume ? lprev[tid] : lower_bound_i32(lst, d.y, (int32_t)lo);
+                    const uint32_t a1 = a0 + lower_bound_i32(lst + a0, d.y - a0, (int32_t)hi);
+                    if (deg <= THREADS) lprev[tid] = a1;
                     substart = d.x + a0;
                     sublen = a1 - a0;
                 }
@@ -215,7 +220,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
         if (!dense) {
             for (uint32_t w = tid; w < cwa; w += THREADS) bits[w] = 0;
             __syncthreads();
-            for_each_product(SET, NOT_DENSE, c0, c1, single_chunk, c0, 0u);
+            for_each_product(SET, NOT_DENSE, c0, c1, single_chunk, c0, 0u, false);
             uint32_t s = 0;
             for (uint32_t w = w0; w < w0 + per && w < cwa; ++w) s += __popc(bits[w]);
             uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(s, scratch, &tot);
@@ -272,8 +277,9 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                 }
                 for (uint32_t t = tid; t < s1 - s0; t += THREADS) acc[t] = Acc(0);
                 __syncthreads();
-                if (dense) for_each_product(ACC, IS_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0);
-                else for_each_product(ACC, NOT_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0);
+                const bool resume = s0 > 0 && deg <= THREADS;
+                if (dense) for_each_product(ACC, IS_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
+                else for_each_product(ACC, NOT_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
                 for (uint32_t t = tid; t < s1 - s0; t += THREADS) c_vals[ob + s0 + t] = (V)acc[t];
                 __syncthreads();
             }
