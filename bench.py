@@ -348,6 +348,31 @@ def run_ours(args):
                                     "tril_speedup_numeric": fnum / phases["numeric"],
                                     "tril_speedup_symbolic_plus_numeric": (fs + fnum) / (phases["symbolic"] + phases["numeric"])}
             del fplan
+            # ---- a half-block product of the local computation: rows of the second half against the
+            # first half of the rows as output columns (an off-diagonal block), full mode
+            bplan = B.spsyrk_plan(a.m, a.n, d_rowptr, d_colidx, d_vals, mode=B.FULL)
+            h = a.m // 2
+            bt = []
+            for it in range(3):
+                e0 = ev()
+                B.spsyrk_plan_set_block(bplan, h, a.m, 0, h)
+                e1 = ev()
+                brp = torch.empty(a.m - h + 1, dtype=torch.int64, device="cuda")
+                bn = B.spsyrk_symbolic(bplan, brp)
+                e2 = ev()
+                bci = torch.empty(max(bn, 1), dtype=torch.int32, device="cuda")
+                bcv = torch.empty(max(bn, 1), dtype=d_vals.dtype, device="cuda")
+                B.spsyrk_numeric(bplan, brp, bci, bcv)
+                e3 = ev()
+                torch.cuda.synchronize()
+                bt.append((e0.elapsed_time(e1), e1.elapsed_time(e2), e2.elapsed_time(e3)))
+                del brp, bci, bcv
+            bw, _ = B.spsyrk_plan_stats(bplan)
+            line["block_variant"] = {"block": f"rows [{h}, {a.m}) x columns [0, {h})", "multiply_adds": bw, "nnz": bn,
+                                     "set_block_ms": float(np.mean([t[0] for t in bt[1:]])),
+                                     "symbolic_ms": float(np.mean([t[1] for t in bt[1:]])),
+                                     "numeric_ms": float(np.mean([t[2] for t in bt[1:]]))}
+            del bplan
         torch.cuda.empty_cache()
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)

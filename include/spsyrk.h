@@ -92,6 +92,23 @@ spsyrk_status_t spsyrk_plan_set_rows(spsyrk_plan_t plan, int64_t row_begin, int6
                                      void *cuda_stream);
 
 /*
+ * spsyrk_plan_set_block - re-target an existing plan to the block
+ *     C[R, S] = A[R, :] * A[S, :]^T,   R = [row_begin, row_end),  S = [col_begin, col_end),
+ * i.e. output rows R restricted to output columns S (rows of A again), without repeating the
+ * transpose.  These are the half-block products of the local computation (Algorithm 2, lines 4
+ * and 6: a row half times the other operand, or all rows times a column half; Section IV-A:
+ * halving along rows is a prefix of the row pointers, halving along columns needs the transpose -
+ * which the plan already holds, so a column range is a contiguous piece of every column list).
+ * The plan's mode still applies: in TRIL mode only j <= i is kept (the cut matters when S overlaps
+ * R: R = S gives the lower triangle of a diagonal block); in FULL mode the whole block is produced.
+ * Column ids of the result stay global (in S); the row pointer is tile-local.  Invalidates any
+ * symbolic result.  Synchronises the stream once.  spsyrk_plan_set_rows is the case S = [0, m).
+ * Errors: INVALID_ARG, CUDA.
+ */
+spsyrk_status_t spsyrk_plan_set_block(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end,
+                                      int64_t col_begin, int64_t col_end, void *cuda_stream);
+
+/*
  * spsyrk_symbolic - count the stored entries of every output row of the plan's range and
  * turn the counts into row pointers.
  *   cnt[i] = #{ j <= i : rows i and j of A share a column }   (TRIL; all j in FULL mode)

@@ -36,6 +36,8 @@ _i64p = ctypes.POINTER(ctypes.c_int64)
 
 _lib.spsyrk_plan.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _vp, _vp, _int, _int, _i64, _i64, _vp, _szp, _vp]
 _lib.spsyrk_plan_set_rows.argtypes = [_vp, _i64, _i64, _vp]
+_lib.spsyrk_plan_set_block.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp]
+_lib.spsyrk_plan_set_block.restype = _int
 _lib.spsyrk_symbolic.argtypes = [_vp, _vp, _i64p, _vp]
 _lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
@@ -143,6 +145,13 @@ def spsyrk_plan(m, n, rowptr, colidx, vals, mode=TRIL, row_begin=0, row_end=None
 
 def spsyrk_plan_set_rows(plan: Plan, row_begin: int, row_end: int, stream=None):
     _check(_lib.spsyrk_plan_set_rows(plan._h, row_begin, row_end, _stream(stream)), "spsyrk_plan_set_rows")
+    plan.row_begin, plan.row_end = row_begin, row_end
+
+
+def spsyrk_plan_set_block(plan: Plan, row_begin: int, row_end: int, col_begin: int, col_end: int, stream=None):
+    """Restrict the plan to output rows [row_begin, row_end) and output columns [col_begin, col_end)."""
+    _check(_lib.spsyrk_plan_set_block(plan._h, row_begin, row_end, col_begin, col_end, _stream(stream)),
+           "spsyrk_plan_set_block")
     plan.row_begin, plan.row_end = row_begin, row_end
 
 

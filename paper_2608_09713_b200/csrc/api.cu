@@ -56,6 +56,9 @@ struct spsyrk_plan_s {
     // workspace views
     int32_t* perm;
     uint4* hdr;  // per-row headers in class order
+    uint2* desc_full;  // descriptors for the whole column range (written by the transpose)
+    uint2* desc_blk;   // descriptors narrowed to the current column range
+    int32_t s0, s1;    // current column range
     int32_t* cnt;
     uint8_t* cls;
     uint32_t* colcnt;
@@ -90,6 +93,7 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     auto at_row = c.take<int32_t>(nnz);
     auto at_val = c.take<char>(nnz * sv);
     auto desc = c.take<uint2>(nnz);
+    auto desc_blk = c.take<uint2>(nnz);
     auto work = c.take<int64_t>(m);
     auto perm = c.take<int32_t>(m);
     auto hdr = c.take<uint4>(m);
@@ -114,6 +118,7 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     if (pl) {
         pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.desc = desc;
         pl->dev.work = work; pl->dev.err = err;
+        pl->desc_full = desc; pl->desc_blk = desc_blk;
         pl->perm = perm; pl->hdr = hdr; pl->cnt = cnt; pl->cls = cls; pl->colcnt = colcnt;
         pl->rx_key_a = rx_key_a; pl->rx_row_a = rx_row_a; pl->rx_pos_a = rx_pos_a; pl->rx_key_b = rx_key_b; pl->rx_row_b = rx_row_b;
         pl->rx_pos_b = rx_pos_b; pl->rx_hist = rx_hist; pl->rx_offsets = rx_offsets;
@@ -137,6 +142,14 @@ void launch_row_expand(spsyrk_plan_s* pl, cudaStream_t st) {
     const PlanDev& P = pl->dev;
     const int64_t threads = (int64_t)P.m * G;
     row_expand_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P.rowptr, P.colidx, P.m, pl->rx_row_b, P.err);
+    note_launches(1);
+}
+
+template <int G>
+void launch_block_desc(spsyrk_plan_s* pl, cudaStream_t st) {
+    const PlanDev& P = pl->dev;
+    const int64_t threads = (int64_t)(P.r1 - P.r0) * G;
+    block_desc_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P, pl->desc_full, pl->desc_blk, pl->s0, pl->s1);
     note_launches(1);
 }
 
@@ -186,9 +199,23 @@ spsyrk_status_t sort_by_column(spsyrk_plan_s* pl, cudaStream_t st) {
 
 // work estimate + binning of the plan's current row range; reads class sizes back (one sync)
 spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
-    const PlanDev& P = pl->dev;
-    const int64_t rows = P.r1 - P.r0;
+    const int64_t rows = pl->dev.r1 - pl->dev.r0;
     pl->have_symbolic = false;
+    // descriptors: the transpose's own for the whole column range, else narrowed to [s0, s1)
+    if (pl->s0 <= 0 && pl->s1 >= pl->dev.m) {
+        pl->dev.desc = pl->desc_full;
+    } else {
+        pl->dev.desc = pl->desc_blk;
+        if (rows > 0 && pl->dev.nnz > 0) {
+            switch (group_width(pl->dev.nnz, pl->dev.m)) {
+                case 4: launch_block_desc<4>(pl, st); break;
+                case 8: launch_block_desc<8>(pl, st); break;
+                case 16: launch_block_desc<16>(pl, st); break;
+                default: launch_block_desc<32>(pl, st); break;
+            }
+        }
+    }
+    const PlanDev& P = pl->dev;
     SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->work_total_dev, 0, sizeof(unsigned long long), st));
     if (rows > 0) {
         switch (group_width(P.nnz, P.m)) {
@@ -349,6 +376,8 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     pl->dtype = dtype;
     pl->rows_cap = m;
     pl->key64 = m > (int64_t(1) << 22);
+    pl->s0 = 0;
+    pl->s1 = (int32_t)m;
     {
         int dev_id = 0;
         pl->sm_count = 148;
@@ -393,11 +422,20 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     return SPSYRK_OK;
 }
 
-spsyrk_status_t spsyrk_plan_set_rows(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end, void* cuda_stream) {
+spsyrk_status_t spsyrk_plan_set_block(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end, int64_t col_begin,
+                                      int64_t col_end, void* cuda_stream) {
     if (!plan || row_begin < 0 || row_end < row_begin || row_end > plan->dev.m) return SPSYRK_ERR_INVALID_ARG;
+    if (col_begin < 0 || col_end < col_begin || col_end > plan->dev.m) return SPSYRK_ERR_INVALID_ARG;
     plan->dev.r0 = (int32_t)row_begin;
     plan->dev.r1 = (int32_t)row_end;
+    plan->s0 = (int32_t)col_begin;
+    plan->s1 = (int32_t)col_end;
     return estimate_and_bin(plan, static_cast<cudaStream_t>(cuda_stream));
+}
+
+spsyrk_status_t spsyrk_plan_set_rows(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end, void* cuda_stream) {
+    if (!plan) return SPSYRK_ERR_INVALID_ARG;
+    return spsyrk_plan_set_block(plan, row_begin, row_end, 0, plan->dev.m, cuda_stream);
 }
 
 spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t* d_c_rowptr, int64_t* nnz_out, void* cuda_stream) {

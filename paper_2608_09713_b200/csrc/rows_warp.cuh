@@ -21,6 +21,12 @@ __host__ __device__ constexpr int numeric_warps(int n) { return n >= 512 ? 2 : n
 // register budget: at least this many CTAs of the numeric kernel must fit on an SM
 __host__ __device__ constexpr int numeric_min_ctas(int n) { return n == 256 ? 6 : 1; }
 
+// lane holding the s-th (0-based) set bit of mask
+__device__ __forceinline__ uint32_t nth_set_lane(unsigned mask, uint32_t s) {
+    for (uint32_t k = 0; k < s; ++k) mask &= mask - 1;
+    return (uint32_t)(__ffs(mask) - 1);
+}
+
 // Asynchronous global -> shared copies of 4 or 8 bytes (no register staging), grouped per thread.
 template <int BYTES>
 __device__ __forceinline__ void cp_async(void* smem_dst, const void* gmem_src) {
@@ -77,11 +83,13 @@ __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) nu
     auto load_a = [&](const uint4& h) { return (uint32_t)lane < h.z ? (Acc) static_cast<const V*>(P.vals)[(int64_t)h.y + lane] : Acc(0); };
     // issue the gathers of one row into buffer b; returns its item count
     auto issue = [&](const uint4& h, const uint2& d, Acc a, int b) -> uint32_t {
-        const bool live = (uint32_t)lane < h.z;
         const uint32_t incl = warp_inclusive_scan(d.y);
         const uint32_t w = __shfl_sync(FULL_MASK, incl, 31);
-        const uint32_t off = live ? incl - d.y : 0xffffffffu;  // first item of this lane's list
-        const uint32_t smo = d.x - off;                        // item t of this list is entry t + smo
+        // a list without items (possible when the plan is restricted to a column range) takes no part
+        const unsigned nzmask = __ballot_sync(FULL_MASK, d.y > 0);
+        const bool gaps = (nzmask & (nzmask + 1u)) != 0;          // the non-empty lists are not lanes 0..k-1
+        const uint32_t off = d.y > 0 ? incl - d.y : 0xffffffffu;  // first item of this lane's list
+        const uint32_t smo = d.x - off;                           // item t of this list is entry t + smo
         s_a[warp][b][lane] = a;
 #pragma unroll
         for (int r = 0; r < R; ++r) {
@@ -91,7 +99,8 @@ __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) nu
                 const uint32_t rel = off - (uint32_t)(r * 32);
                 const uint32_t before = __popc(__ballot_sync(FULL_MASK, off <= (uint32_t)(r * 32)));
                 const uint32_t startbits = __reduce_or_sync(FULL_MASK, (rel - 1u < 31u) ? (1u << rel) : 0u);
-                const uint32_t s = before - 1u + __popc(startbits & (0xfffffffeu >> (31 - lane)));
+                uint32_t s = before - 1u + __popc(startbits & (0xfffffffeu >> (31 - lane)));
+                if (gaps) s = nth_set_lane(nzmask, s & 31);  // s counted non-empty lists: back to a lane
                 const uint32_t q = r * 32 + lane + __shfl_sync(FULL_MASK, smo, s & 31);
                 const uint32_t t = r * 32 + lane;
                 if (t < w) {
@@ -238,10 +247,11 @@ __global__ void __launch_bounds__(symbolic_warps(N) * 32) symbolic_warp_kernel(P
     auto load_hdr = [&](int64_t idx) { return idx < nrows ? hdr[idx] : none; };
     auto load_desc = [&](const uint4& h) { return (uint32_t)lane < h.z ? P.desc[(int64_t)h.y + lane] : make_uint2(0u, 0u); };
     auto issue = [&](const uint4& h, const uint2& d, int b) -> uint32_t {
-        const bool live = (uint32_t)lane < h.z;
         const uint32_t incl = warp_inclusive_scan(d.y);
         const uint32_t w = __shfl_sync(FULL_MASK, incl, 31);
-        const uint32_t off = live ? incl - d.y : 0xffffffffu;
+        const unsigned nzmask = __ballot_sync(FULL_MASK, d.y > 0);
+        const bool gaps = (nzmask & (nzmask + 1u)) != 0;
+        const uint32_t off = d.y > 0 ? incl - d.y : 0xffffffffu;
         const uint32_t smo = d.x - off;
 #pragma unroll
         for (int r = 0; r < R; ++r) {
@@ -249,7 +259,8 @@ __global__ void __launch_bounds__(symbolic_warps(N) * 32) symbolic_warp_kernel(P
                 const uint32_t rel = off - (uint32_t)(r * 32);
                 const uint32_t before = __popc(__ballot_sync(FULL_MASK, off <= (uint32_t)(r * 32)));
                 const uint32_t startbits = __reduce_or_sync(FULL_MASK, (rel - 1u < 31u) ? (1u << rel) : 0u);
-                const uint32_t s = before - 1u + __popc(startbits & (0xfffffffeu >> (31 - lane)));
+                uint32_t s = before - 1u + __popc(startbits & (0xfffffffeu >> (31 - lane)));
+                if (gaps) s = nth_set_lane(nzmask, s & 31);
                 const uint32_t q = r * 32 + lane + __shfl_sync(FULL_MASK, smo, s & 31);
                 if ((uint32_t)(r * 32 + lane) < w) cp_async<4>(&s_j[warp][b][r * 32 + lane], P.at_row + q);
             }

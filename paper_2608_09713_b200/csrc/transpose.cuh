@@ -79,6 +79,26 @@ struct EmitTransposeFinal {
     }
 };
 
+// Restriction of the plan to output columns [s0, s1): column k's entries with row in that range are
+// a contiguous piece of its (row-sorted) list, so the descriptor of every nonzero of the rows
+// [r0, r1) is narrowed to that piece by two binary searches inside its full-range prefix.
+template <int G>
+static __global__ void __launch_bounds__(256) block_desc_kernel(PlanDev P, const uint2* __restrict__ desc_full,
+                                                                uint2* __restrict__ desc_blk, int32_t s0, int32_t s1) {
+    const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    const int gl = threadIdx.x & (G - 1);
+    if (gid >= P.r1 - P.r0) return;
+    const int64_t i = P.r0 + gid;
+    const int64_t p0 = P.rowptr[i], p1 = P.rowptr[i + 1];
+    for (int64_t p = p0 + gl; p < p1; p += G) {
+        const uint2 full = desc_full[p];
+        const int32_t* lst = P.at_row + full.x;
+        const uint32_t lo = s0 <= 0 ? 0u : lower_bound_i32(lst, full.y, s0);
+        const uint32_t hi = lower_bound_i32(lst, full.y, s1);
+        desc_blk[p] = make_uint2(full.x + lo, hi > lo ? hi - lo : 0u);
+    }
+}
+
 // Step a2: per-row work w[i] = sum of the descriptor lengths of row i (G lanes per row), and the
 // class of the row.  Rows of the range [r0, r1) only.
 //   class 0: no work; 1..5: w <= 32, 64, 128, 256, 512 and at most 32 nonzeros (one warp, register sort)

@@ -277,3 +277,56 @@ def test_workspace_and_alignment_errors(B):
     st = B._lib.spsyrk_plan(ctypes.byref(h), a.m, a.n, a.nnz, B._p(rowptr), ctypes.c_void_p(shifted.data_ptr() + 4),
                             B._p(vals), 0, 0, 0, a.m, B._p(ws), ctypes.byref(sz), None)
     assert st == 1                                                      # column ids not 16-byte aligned
+
+
+# ---------------------------------------------------------------- blocks C[R, S] (Algorithm 2, lines 4 and 6)
+def oracle_block(a, mode, r0, r1, s0, s1, cols):
+    """Rows [r0, r1) of the product restricted to columns [s0, s1): the definition, then a column filter."""
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, mode, r0, r1, cols=cols)
+    keep = (ref.colidx >= s0) & (ref.colidx < s1)
+    rows = np.repeat(np.arange(r1 - r0), np.diff(ref.rowptr))
+    rowptr = np.zeros(r1 - r0 + 1, dtype=np.int64)
+    np.cumsum(np.bincount(rows[keep], minlength=r1 - r0), out=rowptr[1:])
+
+    class R:  # same fields as the oracle's result
+        pass
+    out = R()
+    out.rowptr, out.colidx, out.vals, out.absvals = rowptr, ref.colidx[keep], ref.vals[keep], ref.absvals[keep]
+    return out
+
+
+@pytest.mark.parametrize("idx", [2, 3, 4, 5])
+def test_blocks(B, idx):
+    a = W.small(idx)
+    cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
+    d = dev(a)
+    plan = B.spsyrk_plan(a.m, a.n, *d, mode=B.FULL)
+    h = a.m // 2
+    blocks = [(0, h // 2, h, a.m),            # row top half of a lower block x the other operand
+              (h, a.m, h + (a.m - h) // 2, a.m),   # all rows x right half of the columns
+              (h, a.m, 0, h),                 # an off-diagonal block
+              (10, 50, 0, 1),                 # one output column
+              (h, h + 7, 3, 3)]               # empty column range
+    for r0, r1, s0, s1 in blocks:
+        B.spsyrk_plan_set_block(plan, r0, r1, s0, s1)
+        rp, ci, cv, _ = B.tril_syrk(a.m, a.n, *d, plan=plan)
+        ref = oracle_block(a, oracle.FULL, r0, r1, s0, s1, cols)
+        assert np.array_equal(rp.cpu().numpy(), ref.rowptr), (r0, r1, s0, s1)
+        assert np.array_equal(ci.cpu().numpy(), ref.colidx)
+        check_values(cv.cpu().numpy(), ref, a.vals.dtype)
+    # TRIL mode with S = R is the lower triangle of a diagonal block
+    tplan = B.spsyrk_plan(a.m, a.n, *d, mode=B.TRIL)
+    B.spsyrk_plan_set_block(tplan, h, a.m, h, a.m)
+    rp, ci, cv, _ = B.tril_syrk(a.m, a.n, *d, plan=tplan)
+    ref = oracle_block(a, oracle.TRIL, h, a.m, h, a.m, cols)
+    assert np.array_equal(rp.cpu().numpy(), ref.rowptr) and np.array_equal(ci.cpu().numpy(), ref.colidx)
+    check_values(cv.cpu().numpy(), ref, a.vals.dtype)
+    # four blocks tile the full product: entry counts add up
+    B.spsyrk_plan_set_rows(plan, 0, a.m)
+    total = B.tril_syrk(a.m, a.n, *d, plan=plan)[1].numel()
+    parts = 0
+    for r0, r1 in ((0, h), (h, a.m)):
+        for s0, s1 in ((0, h), (h, a.m)):
+            B.spsyrk_plan_set_block(plan, r0, r1, s0, s1)
+            parts += B.tril_syrk(a.m, a.n, *d, plan=plan)[1].numel()
+    assert parts == total
