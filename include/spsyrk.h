@@ -153,6 +153,18 @@ spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
                               void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
 
 /*
+ * spsyrk_symv - y = C x from the stored lower triangle alone,
+ *     C x = C_L x + (x^T C_L)^T - D x        (Section V-F, Eq. 1: the triangular output is consumed
+ * directly, C_L^T is never formed and the diagonal is counted once).  C_L is any lower-triangular
+ * CSR (diagonal included) of F64 or F32 values; d_x[m] and d_y[m] are device vectors of the same
+ * type; y is overwritten.  The reflected contributions are accumulated with atomic adds, so the
+ * last bits of y can differ from run to run.  Asynchronous.  Errors: INVALID_ARG, CUDA.
+ */
+spsyrk_status_t spsyrk_symv(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
+                            const int64_t *d_l_rowptr, const int32_t *d_l_colidx, const void *d_l_vals,
+                            const void *d_x, void *d_y, void *cuda_stream);
+
+/*
  * spsyrk_mirror_rowptr_noalloc - the size step of spsyrk_mirror (step 2: d_f_rowptr[m + 1] and
  * *nnz_full_out of F = C_L + C_L^T - D) for callers that can neither allocate device memory nor
  * pass a workspace.  (The paper has no counterpart: this entry point exists for deployment only.)

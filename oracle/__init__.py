@@ -46,6 +46,8 @@ def _load():
                                          p, p, p, p, p, p]
         lib.oracle_mirror.argtypes = [i64, p, p, p, p, p, p]
         lib.oracle_jaccard.argtypes = [i64, i64, p, p, p, p, p]
+        lib.oracle_symv.argtypes = [i64, p, p, p, p, p, p]
+        lib.oracle_symv.restype = ctypes.c_int
         for f in (lib.oracle_transpose, lib.oracle_syrk_rows, lib.oracle_mirror, lib.oracle_jaccard):
             f.restype = ctypes.c_int
         _lib = lib
@@ -157,3 +159,15 @@ def jaccard(row_begin, rows, a_rowptr, c_rowptr, c_colidx, c_counts) -> np.ndarr
                             _ptr(c_counts), _ptr(jac))
     assert rc == 0
     return jac[:nnz]
+
+
+def symv(m, l_rowptr, l_colidx, l_vals, x):
+    """(y, abs_y): y = C x = C_L x + C_L^T x - D x from the lower triangle; abs_y is the sum of the
+    absolute contributions per row (the scale for rounding comparisons)."""
+    lib = _load()
+    l_rowptr, l_colidx, l_vals, x = _c(l_rowptr, np.int64), _c(l_colidx, np.int32), _c(l_vals, np.float64), _c(x, np.float64)
+    y = np.empty(max(m, 1), dtype=np.float64)
+    ay = np.empty(max(m, 1), dtype=np.float64)
+    rc = lib.oracle_symv(m, _ptr(l_rowptr), _ptr(l_colidx), _ptr(l_vals), _ptr(x), _ptr(y), _ptr(ay))
+    assert rc == 0
+    return y[:m], ay[:m]

@@ -184,3 +184,26 @@ int oracle_jaccard(int64_t row_begin, int64_t rows, const int64_t *a_rowptr,
     }
     return 0;
 }
+
+/* y = C x from the stored lower triangle (Section V-F, Eq. 1): C x = C_L x + (x^T C_L)^T - D x.
+ * Written as the three terms of the equation, each a plain loop; abs_y receives
+ * sum |c_rj x_j| over all contributions of row r, the scale for rounding comparisons. */
+int oracle_symv(int64_t m, const int64_t *l_rowptr, const int32_t *l_colidx, const double *l_vals,
+                const double *x, double *y, double *abs_y)
+{
+    for (int64_t r = 0; r < m; ++r) { y[r] = 0.0; abs_y[r] = 0.0; }
+    for (int64_t r = 0; r < m; ++r)                      /* C_L x */
+        for (int64_t p = l_rowptr[r]; p < l_rowptr[r + 1]; ++p) {
+            y[r] += l_vals[p] * x[l_colidx[p]];
+            abs_y[r] += fabs(l_vals[p] * x[l_colidx[p]]);
+        }
+    for (int64_t r = 0; r < m; ++r)                      /* (x^T C_L)^T */
+        for (int64_t p = l_rowptr[r]; p < l_rowptr[r + 1]; ++p) {
+            y[l_colidx[p]] += l_vals[p] * x[r];
+            abs_y[l_colidx[p]] += fabs(l_vals[p] * x[r]);
+        }
+    for (int64_t r = 0; r < m; ++r)                      /* - D x */
+        for (int64_t p = l_rowptr[r]; p < l_rowptr[r + 1]; ++p)
+            if (l_colidx[p] == r) { y[r] -= l_vals[p] * x[r]; abs_y[r] += fabs(l_vals[p] * x[r]); }
+    return 0;
+}

@@ -43,6 +43,8 @@ _lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_mirror_rowptr_noalloc.argtypes = [_i64, _vp, _vp, _vp, _i64p, _vp]
 _lib.spsyrk_mirror_rowptr_noalloc.restype = _int
+_lib.spsyrk_symv.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.spsyrk_symv.restype = _int
 _lib.spsyrk_jaccard.argtypes = [_i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_plan_stats.argtypes = [_vp, _i64p, _i64p]
 _lib.spsyrk_plan_buffers.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]
@@ -254,6 +256,17 @@ def spsyrk_mirror(m, l_rowptr, l_colidx, l_vals, stream=None, workspace=None, ou
     _check(_lib.spsyrk_mirror(m, nnz_l, code, _p(l_rowptr), _p(l_colidx), _p(l_vals), _p(f_rowptr), _p(f_colidx),
                               _p(f_vals), ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_mirror(fill)")
     return f_rowptr, f_colidx[:nnz.value], f_vals[:nnz.value]
+
+
+def spsyrk_symv(m, l_rowptr, l_colidx, l_vals, x, y=None, stream=None):
+    """y = C x = C_L x + C_L^T x - D x from the lower triangle only (float64 or float32)."""
+    _dev_check(l_rowptr, l_colidx, l_vals, x, y)
+    assert x.dtype == l_vals.dtype and x.numel() == m
+    if y is None:
+        y = torch.empty(m, dtype=x.dtype, device=x.device)
+    _check(_lib.spsyrk_symv(m, l_colidx.numel(), _DTYPE_CODE[l_vals.dtype], _p(l_rowptr), _p(l_colidx), _p(l_vals),
+                            _p(x), _p(y), _stream(stream)), "spsyrk_symv")
+    return y
 
 
 NOALLOC_MAX_ROWS = 1048576

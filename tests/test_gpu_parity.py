@@ -330,3 +330,16 @@ def test_blocks(B, idx):
             B.spsyrk_plan_set_block(plan, r0, r1, s0, s1)
             parts += B.tril_syrk(a.m, a.n, *d, plan=plan)[1].numel()
     assert parts == total
+
+
+# ------------------------------------------------------------------ consuming the triangle (Section V-F)
+@pytest.mark.parametrize("idx", [1, 3, 4, 5])
+def test_symv(B, idx):
+    a = W.small(idx)
+    (rp, ci, cv), ref, _ = run_and_compare(B, a, 0)
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal(a.m).astype(a.vals.dtype)
+    y = B.spsyrk_symv(a.m, rp, ci, cv, torch.from_numpy(x).cuda()).cpu().numpy()
+    exp, scale = oracle.symv(a.m, rp.cpu().numpy(), ci.cpu().numpy(), cv.cpu().numpy().astype(np.float64), x.astype(np.float64))
+    tol = 1e-12 if a.vals.dtype == np.float64 else 2e-5
+    assert np.all(np.abs(y.astype(np.float64) - exp) <= tol * (scale + 1e-300))

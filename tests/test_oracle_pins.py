@@ -374,3 +374,27 @@ def test_jaccard_identical_rows_give_one():
     assert lookup[(1, 0)] == 1.0
     assert lookup[(2, 0)] == np.float32(1) / np.float32(3)
     assert (3, 0) not in lookup
+
+
+# -------------------------------------------------------------------- triangular SpMV
+def test_symv_equals_a_at_x(small_case):
+    """Section V-F: C x from the lower triangle equals A (A^T x), and equals scipy's product with the
+    mirrored matrix."""
+    _, a, _, tril = small_case
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal(a.m)
+    y, ay = oracle.symv(a.m, tril.rowptr, tril.colidx, tril.vals, x)
+    A = sp.csr_matrix((a.vals.astype(np.float64), a.colidx, a.rowptr), shape=(a.m, a.n))
+    ref = A @ (A.T @ x)
+    absA = abs(A)
+    bound = absA @ (absA.T @ np.abs(x)) + 1e-300
+    assert np.all(np.abs(y - ref) <= 1e-12 * bound)
+    f_rowptr, f_colidx, f_vals = oracle.mirror(a.m, tril.rowptr, tril.colidx, tril.vals)
+    F = sp.csr_matrix((f_vals, f_colidx, f_rowptr), shape=(a.m, a.m))
+    assert np.all(np.abs(y - F @ x) <= 1e-13 * (ay + 1e-300))
+
+
+def test_symv_tiny_by_hand():
+    # C_L = [[5], [., 9], [14, ., 42]], x = (1, 2, 3): C x = (5 + 42, 18, 14 + 126)
+    y, _ = oracle.symv(3, [0, 1, 2, 4], [0, 1, 0, 2], [5.0, 9.0, 14.0, 42.0], [1.0, 2.0, 3.0])
+    assert list(y) == [47.0, 18.0, 140.0]
