@@ -243,7 +243,7 @@ void launch_symbolic_warp(spsyrk_plan_s* pl, int c, cudaStream_t st) {
     const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
     if (count <= 0) return;
     constexpr int SW = symbolic_warps(N);
-    auto kern = symbolic_warp_kernel<N>;
+    auto kern = pl->dev.desc == pl->desc_blk ? symbolic_warp_kernel<N, true> : symbolic_warp_kernel<N, false>;
     int per_sm = 1;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, SW * 32, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
     const int64_t want = (count + SW - 1) / SW;
@@ -259,7 +259,7 @@ void launch_numeric_warp(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int3
     constexpr int NW = numeric_warps(N);
     // persistent warps: exactly as many CTAs as are resident at once, each warp walks its rows with
     // a stride of the whole grid
-    auto kern = numeric_warp_kernel<V, N, Key>;
+    auto kern = pl->dev.desc == pl->desc_blk ? numeric_warp_kernel<V, N, Key, true> : numeric_warp_kernel<V, N, Key, false>;
     int per_sm = 1;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
     const int64_t want = (count + NW - 1) / NW;

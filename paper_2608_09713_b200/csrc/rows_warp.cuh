@@ -54,7 +54,8 @@ __global__ void __launch_bounds__(256) row_header_kernel(PlanDev P, const int32_
 // while row n is sorted and written, the column-list entries of row n+1 stream into shared memory
 // through cp.async, the descriptors of row n+2 and the header of row n+3 are in flight in
 // registers.  Memory latency is hidden inside the warp instead of by occupancy.
-template <typename V, int N, typename Key>
+// GAPS: descriptors may have zero length (plan restricted to a column range)
+template <typename V, int N, typename Key, bool GAPS>
 __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows,
                                                                       const int64_t* __restrict__ c_rowptr,
                                                                       int32_t* __restrict__ c_colidx, V* __restrict__ c_vals) {
@@ -86,8 +87,8 @@ __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) nu
         const uint32_t incl = warp_inclusive_scan(d.y);
         const uint32_t w = __shfl_sync(FULL_MASK, incl, 31);
         // a list without items (possible when the plan is restricted to a column range) takes no part
-        const unsigned nzmask = __ballot_sync(FULL_MASK, d.y > 0);
-        const bool gaps = (nzmask & (nzmask + 1u)) != 0;          // the non-empty lists are not lanes 0..k-1
+        const unsigned nzmask = GAPS ? __ballot_sync(FULL_MASK, d.y > 0) : 0u;
+        const bool gaps = GAPS && (nzmask & (nzmask + 1u)) != 0;  // the non-empty lists are not lanes 0..k-1
         const uint32_t off = d.y > 0 ? incl - d.y : 0xffffffffu;  // first item of this lane's list
         const uint32_t smo = d.x - off;                           // item t of this list is entry t + smo
         s_a[warp][b][lane] = a;
@@ -229,7 +230,7 @@ __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) nu
 // (header, descriptors and column-list row ids of later rows in flight while a row is counted), but
 // only the row ids are gathered and they go into a per-warp hash set; the count is the number of
 // successful inserts.
-template <int N>
+template <int N, bool GAPS>
 __global__ void __launch_bounds__(symbolic_warps(N) * 32) symbolic_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows,
                                                                        int32_t* __restrict__ cnt) {
     constexpr int SW = symbolic_warps(N);
@@ -249,8 +250,8 @@ __global__ void __launch_bounds__(symbolic_warps(N) * 32) symbolic_warp_kernel(P
     auto issue = [&](const uint4& h, const uint2& d, int b) -> uint32_t {
         const uint32_t incl = warp_inclusive_scan(d.y);
         const uint32_t w = __shfl_sync(FULL_MASK, incl, 31);
-        const unsigned nzmask = __ballot_sync(FULL_MASK, d.y > 0);
-        const bool gaps = (nzmask & (nzmask + 1u)) != 0;
+        const unsigned nzmask = GAPS ? __ballot_sync(FULL_MASK, d.y > 0) : 0u;
+        const bool gaps = GAPS && (nzmask & (nzmask + 1u)) != 0;
         const uint32_t off = d.y > 0 ? incl - d.y : 0xffffffffu;
         const uint32_t smo = d.x - off;
 #pragma unroll
