@@ -175,19 +175,32 @@ __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) nu
         // order; repeat while a lane that is one single run passes a changed sum on (almost never)
         const bool joins = same[0] && key[0] != PAD;
         if (__any_sync(FULL_MASK, joins)) {
-            for (int iter = 0; iter < 32; ++iter) {
+            // a leading run of three or more (or, with one or two keys per lane, possibly the whole lane)
+            const bool deep = joins && (R >= 3 ? (same[1] && same[R >= 3 ? 2 : 0]) : true);
+            if (!__any_sync(FULL_MASK, deep)) {
+                // common case: the run reaches at most two elements into the lane, so no lane's last
+                // sum changes and one step settles everything
                 const Acc carry = __shfl_up_sync(FULL_MASK, sum[R - 1], 1);
-                const Acc old_tail = sum[R - 1];
                 if (joins) {
-                    Acc acc = carry;
-                    bool in_run = true;
-#pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        in_run = in_run && (r == 0 || same[r]);
-                        if (in_run) { acc = acc_add(acc, s_v[warp][b][(uint32_t)(key[r] & (Key)(N - 1))]); sum[r] = acc; }
-                    }
+                    const Acc a0 = acc_add(carry, s_v[warp][b][(uint32_t)(key[0] & (Key)(N - 1))]);
+                    sum[0] = a0;
+                    if (R >= 2 && same[R >= 2 ? 1 : 0]) sum[R >= 2 ? 1 : 0] = acc_add(a0, s_v[warp][b][(uint32_t)(key[R >= 2 ? 1 : 0] & (Key)(N - 1))]);
                 }
-                if (!__any_sync(FULL_MASK, joins && !(sum[R - 1] == old_tail))) break;
+            } else {
+                for (int iter = 0; iter < 32; ++iter) {
+                    const Acc carry = __shfl_up_sync(FULL_MASK, sum[R - 1], 1);
+                    const Acc old_tail = sum[R - 1];
+                    if (joins) {
+                        Acc acc = carry;
+                        bool in_run = true;
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            in_run = in_run && (r == 0 || same[r]);
+                            if (in_run) { acc = acc_add(acc, s_v[warp][b][(uint32_t)(key[r] & (Key)(N - 1))]); sum[r] = acc; }
+                        }
+                    }
+                    if (!__any_sync(FULL_MASK, joins && !(sum[R - 1] == old_tail))) break;
+                }
             }
         }
         __syncwarp();  // every lane has read its products: the buffer is free for the output
