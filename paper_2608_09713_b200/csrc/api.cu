@@ -24,6 +24,7 @@ constexpr uint32_t ROW_CHUNK_BITS_MAX_NUMERIC = 1u << 18;
 constexpr uint32_t ROW_CHUNK_BITS_MAX_SYMBOLIC = 1u << 20;
 constexpr int TRANSPOSE_RADIX_BITS = 8;
 constexpr size_t LARGE_SMEM_BUDGET = 200 * 1024;
+constexpr int GLOBAL_ACC_CTAS = 160;  // upper bound of the persistent heavy-row grid (one CTA per SM)
 constexpr uint32_t BLOCK_ACC_SLOTS = 4096;
 
 size_t dtype_size(spsyrk_dtype_t t) { return t == SPSYRK_F64 ? 8 : 4; }
@@ -71,6 +72,9 @@ struct spsyrk_plan_s {
     int64_t* partials;
     int64_t* class_start_dev;  // NCLASS + 1
     unsigned long long* work_total_dev;
+    uint32_t* row_counter;  // row dispenser of the persistent heavy-row kernel
+    double* gacc;           // its global accumulator slices (GLOBAL_ACC_CTAS x gslots, 8 bytes per slot)
+    uint32_t gslots;
     // host facts
     int64_t class_start[NCLASS + 1];
     int64_t work_total;
@@ -115,7 +119,12 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     auto class_start_dev = c.take<int64_t>(NCLASS + 1);
     auto work_total_dev = c.take<unsigned long long>(1);
     auto err = c.take<uint32_t>(1);
+    auto row_counter = c.take<uint32_t>(1);
+    // one global accumulator slice per persistent CTA of the heavy-row numeric kernel
+    const uint32_t gslots = pow2_at_least((uint64_t)std::max<int64_t>(m, 1), 1024u, ROW_CHUNK_BITS_MAX_NUMERIC);
+    auto gacc = c.take<double>((size_t)GLOBAL_ACC_CTAS * gslots);
     if (pl) {
+        pl->row_counter = row_counter; pl->gacc = gacc; pl->gslots = gslots;
         pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.desc = desc;
         pl->dev.work = work; pl->dev.err = err;
         pl->desc_full = desc; pl->desc_blk = desc_blk;
@@ -301,7 +310,8 @@ spsyrk_status_t launch_symbolic_cta(spsyrk_plan_s* pl, int c, cudaStream_t st) {
     const size_t smem = CtaRowSmem<int32_t, THREADS, false>::bytes(cb, 0);
     auto kern = rows_cta_kernel<int32_t, THREADS, false>;
     SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, 0u, pl->cnt, nullptr, nullptr, nullptr);
+    kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, 0u, pl->cnt, nullptr, nullptr, nullptr,
+                                                  0u, nullptr, nullptr, 0u);
     note_launches(1);
     return SPSYRK_OK;
 }
@@ -322,9 +332,23 @@ spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_
     const size_t smem = CtaRowSmem<V, THREADS, true>::bytes(cb, slots);
     auto kern = rows_cta_kernel<V, THREADS, true>;
     SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    // rows that overflow the shared-memory tile go to the persistent variant with global accumulators
+    const bool use_global = acc_slots_or_zero == 0 && pl->gslots >= cb;
+    const uint32_t gslots = use_global ? pl->gslots : 0u;
     kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, c_rowptr, c_colidx,
-                                                  static_cast<V*>(c_vals));
+                                                  static_cast<V*>(c_vals), 0u, nullptr, nullptr, gslots);
     note_launches(1);
+    if (use_global) {
+        auto gkern = rows_cta_kernel<V, THREADS, true, true>;
+        const size_t gsmem = CtaRowSmem<V, THREADS, true>::bytes(cb, 0);
+        SPSYRK_CUDA_TRY(cudaFuncSetAttribute(gkern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gsmem));
+        SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->row_counter, 0, sizeof(uint32_t), st));
+        const unsigned grid = (unsigned)std::min<int64_t>(std::min<int64_t>(pl->sm_count, GLOBAL_ACC_CTAS), count);
+        gkern<<<grid, THREADS, gsmem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, c_rowptr, c_colidx,
+                                            static_cast<V*>(c_vals), (uint32_t)count, pl->row_counter,
+                                            reinterpret_cast<Acc*>(pl->gacc), gslots);
+        note_launches(1);
+    }
     return SPSYRK_OK;
 }
 

@@ -30,13 +30,21 @@ struct CtaRowSmem {
     }
 };
 
-template <typename V, int THREADS, bool NUMERIC>
+// GLOBAL_ACC: the variant for rows whose output does not fit the shared-memory accumulator tile.
+// Instead of walking the lists once per tile, it accumulates the whole row in one pass into a
+// global-memory slice owned by the CTA (global atomics, served by L2).  It runs as a persistent grid:
+// CTAs fetch rows from a counter, so that the slice indexed by blockIdx.x is never shared.  The
+// two variants are launched over the same row list and each skips the rows of the other.
+template <typename V, int THREADS, bool NUMERIC, bool GLOBAL_ACC = false>
 __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int32_t* __restrict__ rows,
                                                            uint32_t chunk_bits, uint32_t acc_slots,
                                                            int32_t* __restrict__ cnt,
                                                            const int64_t* __restrict__ c_rowptr,
-                                                           int32_t* __restrict__ c_colidx, V* __restrict__ c_vals) {
+                                                           int32_t* __restrict__ c_colidx, V* __restrict__ c_vals,
+                                                           uint32_t nrows = 0, uint32_t* row_counter = nullptr,
+                                                           typename AccOf<V>::type* gscratch = nullptr, uint32_t gslots = 0) {
     using Acc = typename AccOf<V>::type;
+    __shared__ uint32_t s_row;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ uint32_t scratch[33];
     __shared__ uint32_t s_sel[2];
@@ -52,13 +60,20 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     size_t words = (size_t)cw * (NUMERIC ? 2 : 1) + 5 * THREADS + 1;
     words = (words + 3) & ~size_t(3);
     Acc* la = reinterpret_cast<Acc*>(smem_raw + words * 4);
-    Acc* acc = la + THREADS;
+    Acc* acc = GLOBAL_ACC ? gscratch + (size_t)blockIdx.x * gslots : la + THREADS;
+    const uint32_t tile_slots = GLOBAL_ACC ? gslots : acc_slots;  // slots accumulated per pass over the lists
 
     const int tid = threadIdx.x;
-    // later rows carry longer column prefixes: hand them out first so that the tail of the launch is light
-    const int32_t rloc = rows[gridDim.x - 1 - blockIdx.x];
+    auto do_row = [&](const int32_t rloc) {
     const int64_t i = (int64_t)P.r0 + rloc;
     const uint32_t U = P.mode == SPSYRK_TRIL ? (uint32_t)i + 1u : (uint32_t)P.m;
+    if (NUMERIC) {
+        // rows that overflow the shared-memory tile (and are not full) belong to the global variant
+        const int64_t row_cnt = c_rowptr[rloc + 1] - c_rowptr[rloc];
+        const bool wants_global = gslots > 0 && row_cnt > (int64_t)acc_slots && U <= chunk_bits && row_cnt < (int64_t)U &&
+                                  row_cnt <= (int64_t)gslots;
+        if (wants_global != GLOBAL_ACC) return;
+    }
     const int64_t p0 = P.rowptr[i];
     const uint32_t deg = (uint32_t)(P.rowptr[i + 1] - p0);
     const int64_t out_base = NUMERIC ? c_rowptr[rloc] : 0;
@@ -245,8 +260,8 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     }
                 }
             }
-            for (uint32_t s0 = 0; s0 < tot; s0 += acc_slots) {
-                const uint32_t s1 = min(s0 + acc_slots, tot);
+            for (uint32_t s0 = 0; s0 < tot; s0 += tile_slots) {
+                const uint32_t s1 = min(s0 + tile_slots, tot);
                 const bool single_tile = (s0 == 0 && s1 == tot);
                 uint32_t jlo = c0, jhi = c1;
                 if (!single_tile && dense) {
@@ -280,7 +295,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                 const bool resume = s0 > 0 && deg <= THREADS;
                 if (dense) for_each_product(ACC, IS_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
                 else for_each_product(ACC, NOT_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
-                for (uint32_t t = tid; t < s1 - s0; t += THREADS) c_vals[ob + s0 + t] = (V)acc[t];
+                for (uint32_t t = tid; t < s1 - s0; t += THREADS) c_vals[ob + s0 + t] = (V)(GLOBAL_ACC ? __ldcg(acc + t) : acc[t]);
                 __syncthreads();
             }
         }
@@ -288,6 +303,22 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
         __syncthreads();
     }
     if (!NUMERIC && tid == 0) cnt[rloc] = (int32_t)total_cnt;
+    };  // do_row
+
+    if (GLOBAL_ACC) {
+        for (;;) {
+            if (tid == 0) s_row = atomicAdd(row_counter, 1u);
+            __syncthreads();
+            const uint32_t r = s_row;
+            __syncthreads();
+            if (r >= nrows) break;
+            do_row(rows[nrows - 1 - r]);
+            __syncthreads();
+        }
+    } else {
+        // later rows carry longer column prefixes: hand them out first so that the tail of the launch is light
+        do_row(rows[gridDim.x - 1 - blockIdx.x]);
+    }
 }
 
 }  // namespace spsyrk
