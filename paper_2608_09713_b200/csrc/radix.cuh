@@ -5,8 +5,8 @@
 //
 // One pass = three launches: per-tile digit histogram, device-wide scan of the digit-major
 // histogram, scatter.  In the scatter a warp owns a contiguous slice of the tile and ranks its
-// elements 32 at a time with __match_any_sync (elements with equal digits find each other, the
-// lowest lane bumps the warp's counter), an exclusive prefix over the warps makes the ranks
+// elements 32 at a time (elements with equal digits find each other through one warp vote per digit
+// bit, the lowest lane bumps the warp's counter), an exclusive prefix over the warps makes the ranks
 // tile-wide and stable, the tile is reordered digit-major in shared memory and written out in
 // runs.  There is no waiting between CTAs.
 #pragma once
@@ -119,7 +119,15 @@ __global__ void __launch_bounds__(RX_THREADS) radix_scatter_kernel(const uint32_
         const int t = warp * RX_CHUNK + i * 32 + lane;
         const bool valid = t < tile_n;
         const uint32_t d = valid ? ((s_key[t] >> shift) & (NB - 1)) : 0u;
-        const unsigned peers = __match_any_sync(FULL_MASK, valid ? d : (uint32_t)(NB + lane));
+        // lanes with the same digit, found one bit at a time with warp votes (cheaper here than the
+        // match instruction, whose unit saturates long before memory does)
+        unsigned peers = __ballot_sync(FULL_MASK, valid);
+#pragma unroll
+        for (int b = 0; b < BITS; ++b) {
+            const bool bit = (d >> b) & 1u;
+            const unsigned bal = __ballot_sync(FULL_MASK, bit);
+            peers &= bit ? bal : ~bal;
+        }
         const int leader = __ffs(peers) - 1;
         uint32_t prev = 0;
         if (valid && lane == leader) {
