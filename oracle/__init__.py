@@ -47,6 +47,8 @@ def _load():
         lib.oracle_mirror.argtypes = [i64, p, p, p, p, p, p]
         lib.oracle_jaccard.argtypes = [i64, i64, p, p, p, p, p]
         lib.oracle_symv.argtypes = [i64, p, p, p, p, p, p]
+        lib.oracle_column_panel.argtypes = [i64, p, p, p, i64, i64, p, p, p]
+        lib.oracle_add.argtypes = [i64, p, p, p, p, p, p, p, p, p]
         lib.oracle_symv.restype = ctypes.c_int
         for f in (lib.oracle_transpose, lib.oracle_syrk_rows, lib.oracle_mirror, lib.oracle_jaccard):
             f.restype = ctypes.c_int
@@ -171,3 +173,36 @@ def symv(m, l_rowptr, l_colidx, l_vals, x):
     rc = lib.oracle_symv(m, _ptr(l_rowptr), _ptr(l_colidx), _ptr(l_vals), _ptr(x), _ptr(y), _ptr(ay))
     assert rc == 0
     return y[:m], ay[:m]
+
+
+def column_panel(m, rowptr, colidx, vals, k0, k1):
+    """A(:, [k0, k1)) as CSR with unchanged column ids (rowptr int64, colidx int32, vals float64)."""
+    lib = _load()
+    rowptr, colidx, vals = _c(rowptr, np.int64), _c(colidx, np.int32), _c(vals, np.float64)
+    out_rowptr = np.empty(m + 1, dtype=np.int64)
+    rc = lib.oracle_column_panel(m, _ptr(rowptr), _ptr(colidx), _ptr(vals), k0, k1, _ptr(out_rowptr), None, None)
+    assert rc == 0
+    nnz = int(out_rowptr[m])
+    out_colidx = np.empty(max(nnz, 1), dtype=np.int32)
+    out_vals = np.empty(max(nnz, 1), dtype=np.float64)
+    rc = lib.oracle_column_panel(m, _ptr(rowptr), _ptr(colidx), _ptr(vals), k0, k1, _ptr(out_rowptr),
+                                 _ptr(out_colidx), _ptr(out_vals))
+    assert rc == 0
+    return out_rowptr, out_colidx[:nnz], out_vals[:nnz]
+
+
+def add(m, x_rowptr, x_colidx, x_vals, y_rowptr, y_colidx, y_vals):
+    """Z = X + Y on sorted CSR rows: union structure, x + y where both store the entry."""
+    lib = _load()
+    x_rowptr, x_colidx, x_vals = _c(x_rowptr, np.int64), _c(x_colidx, np.int32), _c(x_vals, np.float64)
+    y_rowptr, y_colidx, y_vals = _c(y_rowptr, np.int64), _c(y_colidx, np.int32), _c(y_vals, np.float64)
+    z_rowptr = np.empty(m + 1, dtype=np.int64)
+    args = (m, _ptr(x_rowptr), _ptr(x_colidx), _ptr(x_vals), _ptr(y_rowptr), _ptr(y_colidx), _ptr(y_vals))
+    rc = lib.oracle_add(*args, _ptr(z_rowptr), None, None)
+    assert rc == 0, "rows must be strictly ascending in column"
+    nnz = int(z_rowptr[m])
+    z_colidx = np.empty(max(nnz, 1), dtype=np.int32)
+    z_vals = np.empty(max(nnz, 1), dtype=np.float64)
+    rc = lib.oracle_add(*args, _ptr(z_rowptr), _ptr(z_colidx), _ptr(z_vals))
+    assert rc == 0
+    return z_rowptr, z_colidx[:nnz], z_vals[:nnz]

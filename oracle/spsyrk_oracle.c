@@ -10,6 +10,8 @@
  *   - Section III-A (diagonal processes) and Algorithm 2 line 2: only the lower triangle
  *     is computed.  Section V-F: the stored half includes the diagonal and
  *     C = C_L + C_L^T - D.
+ *   - Section III-A (C_ii = sum over s of SYRK(A_is)) and the "+=" of Algorithm 2: column panels
+ *     of A and the sparse sum that accumulates their products.
  *   - Section III-C: one addition per partial product; the multiply-add count of A A^T is
  *     sum_k nnz(A(:,k))^2.
  *
@@ -205,5 +207,55 @@ int oracle_symv(int64_t m, const int64_t *l_rowptr, const int32_t *l_colidx, con
     for (int64_t r = 0; r < m; ++r)                      /* - D x */
         for (int64_t p = l_rowptr[r]; p < l_rowptr[r + 1]; ++p)
             if (l_colidx[p] == r) { y[r] -= l_vals[p] * x[r]; abs_y[r] += fabs(l_vals[p] * x[r]); }
+    return 0;
+}
+
+/* Column panel A_s = A(:, [k0, k1)) as CSR with the column ids unchanged (Section III-A: the
+ * diagonal block of C is a sum over s of SYRK(A_is), one term per column panel).  Rows keep
+ * their order.  First call with out_colidx == NULL fills out_rowptr[m+1]; second call fills
+ * the entries.  Returns 0. */
+int oracle_column_panel(int64_t m, const int64_t *rowptr, const int32_t *colidx, const double *vals,
+                        int64_t k0, int64_t k1, int64_t *out_rowptr, int32_t *out_colidx, double *out_vals)
+{
+    int64_t o = 0;
+    for (int64_t i = 0; i < m; ++i) {
+        if (!out_colidx) out_rowptr[i] = o;
+        for (int64_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+            if (colidx[p] < k0 || colidx[p] >= k1) continue;
+            if (out_colidx) { out_colidx[o] = colidx[p]; out_vals[o] = vals[p]; }
+            ++o;
+        }
+    }
+    if (!out_colidx) out_rowptr[m] = o;
+    return 0;
+}
+
+/* Z = X + Y for two CSR matrices with rows sorted by column (the "+=" of Algorithm 2 line 2:
+ * the running sum X takes one more panel product Y).  The structure of Z is the union of the
+ * two structures; an entry stored in both gets x + y (one rounded addition, X's value first),
+ * an entry stored in one keeps its value.  Rows of Z are ascending in column.  First call with
+ * z_colidx == NULL fills z_rowptr[m+1]; second call fills the entries.  Returns 0, or -2 if a
+ * row of X or Y is not strictly ascending. */
+int oracle_add(int64_t m, const int64_t *x_rowptr, const int32_t *x_colidx, const double *x_vals,
+               const int64_t *y_rowptr, const int32_t *y_colidx, const double *y_vals,
+               int64_t *z_rowptr, int32_t *z_colidx, double *z_vals)
+{
+    int64_t o = 0;
+    for (int64_t i = 0; i < m; ++i) {
+        int64_t p = x_rowptr[i], pe = x_rowptr[i + 1], q = y_rowptr[i], qe = y_rowptr[i + 1];
+        for (int64_t t = p + 1; t < pe; ++t) if (x_colidx[t] <= x_colidx[t - 1]) return -2;
+        for (int64_t t = q + 1; t < qe; ++t) if (y_colidx[t] <= y_colidx[t - 1]) return -2;
+        if (!z_colidx) z_rowptr[i] = o;
+        while (p < pe || q < qe) {
+            int32_t j;
+            double v;
+            if (q >= qe || (p < pe && x_colidx[p] < y_colidx[q])) { j = x_colidx[p]; v = x_vals[p]; ++p; }
+            else if (p >= pe || y_colidx[q] < x_colidx[p]) { j = y_colidx[q]; v = y_vals[q]; ++q; }
+            else { j = x_colidx[p]; v = x_vals[p] + y_vals[q]; ++p; ++q; }
+            if (z_colidx) { z_colidx[o] = j; z_vals[o] = v; }
+            ++o;
+        }
+    }
+    if (!z_colidx) z_rowptr[m] = o;
     return 0;
 }

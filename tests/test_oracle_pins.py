@@ -398,3 +398,93 @@ def test_symv_tiny_by_hand():
     # C_L = [[5], [., 9], [14, ., 42]], x = (1, 2, 3): C x = (5 + 42, 18, 14 + 126)
     y, _ = oracle.symv(3, [0, 1, 2, 4], [0, 1, 0, 2], [5.0, 9.0, 14.0, 42.0], [1.0, 2.0, 3.0])
     assert list(y) == [47.0, 18.0, 140.0]
+
+
+# ------------------------------------------------- accumulating form over column panels
+def dense_add_reference(x, sx, y, sy):
+    """Dense statement of Z = X + Y with explicit structure masks: stored iff stored in either."""
+    rows = []
+    for i in range(x.shape[0]):
+        out = []
+        for j in range(x.shape[1]):
+            if sx[i, j] and sy[i, j]:
+                out.append((j, x[i, j] + y[i, j]))
+            elif sx[i, j]:
+                out.append((j, x[i, j]))
+            elif sy[i, j]:
+                out.append((j, y[i, j]))
+        rows.append(out)
+    return rows
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_add_dense_brute_force(seed):
+    """Pin: the definition of a sparse sum evaluated entry by entry on dense arrays, with stored
+    zeros on both sides and values that cancel (the entry stays stored)."""
+    rng = np.random.default_rng(100 + seed)
+    m, n = 13, 17
+    x = rng.integers(-2, 3, size=(m, n)).astype(np.float64)
+    y = rng.integers(-2, 3, size=(m, n)).astype(np.float64)
+    sx, sy = rng.random((m, n)) < 0.3, rng.random((m, n)) < 0.3
+    sx[3], sy[5], sx[7], sy[7] = False, False, False, False  # empty rows on either side and on both
+    cx, cy = csr_from_dense(x, sx), csr_from_dense(y, sy)
+    zr, zc, zv = oracle.add(m, cx.rowptr, cx.colidx, cx.vals, cy.rowptr, cy.colidx, cy.vals)
+    ref = dense_add_reference(x, sx, y, sy)
+    for i in range(m):
+        assert list(zip(zc[zr[i]:zr[i + 1]], zv[zr[i]:zr[i + 1]])) == ref[i]
+    assert zr[m] == (sx | sy).sum()
+
+
+def test_add_matches_scipy_on_positive_values():
+    """Pin: scipy's CSR addition (third party); positive values, so it prunes nothing."""
+    rng = np.random.default_rng(7)
+    x = sp.random(200, 300, density=0.05, random_state=rng, format="csr", data_rvs=lambda k: rng.random(k) + 0.5)
+    y = sp.random(200, 300, density=0.08, random_state=rng, format="csr", data_rvs=lambda k: rng.random(k) + 0.5)
+    x.sort_indices(); y.sort_indices()
+    zr, zc, zv = oracle.add(200, x.indptr, x.indices, x.data, y.indptr, y.indices, y.data)
+    z = (x + y).tocsr()
+    z.sort_indices()
+    assert np.array_equal(zr, z.indptr) and np.array_equal(zc, z.indices)
+    assert np.array_equal(zv, z.data)  # one addition per shared entry on both sides
+
+
+def test_add_rejects_unsorted_rows():
+    rowptr = np.array([0, 2], dtype=np.int64)
+    bad = np.array([3, 1], dtype=np.int32)
+    ok = np.array([1, 3], dtype=np.int32)
+    v = np.ones(2)
+    with pytest.raises(AssertionError):
+        oracle.add(1, rowptr, bad, v, rowptr, ok, v)
+
+
+def test_column_panel_matches_scipy_slice(small_case):
+    """Pin: scipy column slicing (third party) for the panel's structure and values."""
+    _, a, _, _ = small_case
+    s = sp.csr_matrix((a.vals.astype(np.float64), a.colidx, a.rowptr), shape=(a.m, a.n))
+    for k0, k1 in [(0, a.n), (0, a.n // 3), (a.n // 3, a.n // 3), (a.n // 3, a.n - 1), (a.n - 1, a.n)]:
+        pr, pc, pv = oracle.column_panel(a.m, a.rowptr, a.colidx, a.vals, k0, k1)
+        ref = s[:, k0:k1].tocsr()
+        ref.sort_indices()
+        assert np.array_equal(pr, ref.indptr)
+        assert np.array_equal(pc, ref.indices + k0)
+        assert np.array_equal(pv, ref.data)
+
+
+@pytest.mark.parametrize("npanels", [1, 2, 5])
+def test_panel_products_sum_to_the_whole(small_case, npanels):
+    """Pin: Section III-A, C_ii = sum_s SYRK(A_is).  The union of the panel structures is the
+    structure of tril(A A^T) exactly; the values agree to rounding (exactly for integer-valued
+    inputs, where every partial sum is exact)."""
+    cfg, a, _, tril = small_case
+    edges = np.linspace(0, a.n, npanels + 1).astype(np.int64)
+    acc = (np.zeros(a.m + 1, dtype=np.int64), np.zeros(0, dtype=np.int32), np.zeros(0))
+    for s in range(npanels):
+        pr, pc, pv = oracle.column_panel(a.m, a.rowptr, a.colidx, a.vals, int(edges[s]), int(edges[s + 1]))
+        t = oracle.syrk(a.m, a.n, pr, pc, pv, oracle.TRIL)
+        acc = oracle.add(a.m, *acc, t.rowptr, t.colidx, t.vals)
+    zr, zc, zv = acc
+    assert np.array_equal(zr, tril.rowptr) and np.array_equal(zc, tril.colidx)
+    if cfg in (2, 4):  # integer-valued inputs
+        assert np.array_equal(zv, tril.vals)
+    else:
+        assert np.all(np.abs(zv - tril.vals) <= 1e-13 * tril.absvals)
