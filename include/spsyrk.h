@@ -153,6 +153,48 @@ spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
                               void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
 
 /*
+ * spsyrk_column_panel - A_s = A(:, [k0, k1)) as CSR, column ids and row order unchanged.
+ * The diagonal block of the product is a sum of rank-k updates, one per column panel of A
+ * (Section III-A: C_ii = sum over s of SYRK(A_is)); this call cuts one panel out of a canonical
+ * CSR matrix so that it can be planned and multiplied on its own.
+ *
+ * Three-step use:
+ *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for m.
+ *   2. d_p_colidx == NULL: writes d_p_rowptr[m + 1] and *nnz_out (synchronises).
+ *   3. all pointers set: fills d_p_colidx / d_p_vals using the d_p_rowptr of step 2.  Asynchronous.
+ * All pointers are device pointers except nnz_out and workspace_bytes (host); nothing is owned
+ * by the library.  nnz = d_rowptr[m].  Requires 0 <= k0 <= k1.  Errors: INVALID_ARG, WORKSPACE, CUDA.
+ */
+spsyrk_status_t spsyrk_column_panel(int64_t m, int64_t nnz, spsyrk_dtype_t dtype,
+                                    const int64_t *d_rowptr, const int32_t *d_colidx, const void *d_vals,
+                                    int64_t k0, int64_t k1,
+                                    int64_t *d_p_rowptr, int32_t *d_p_colidx, void *d_p_vals,
+                                    int64_t *nnz_out,
+                                    void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
+
+/*
+ * spsyrk_accumulate - Z = X + Y for two CSR matrices of m rows whose rows are ascending in column:
+ * the "+=" of Algorithm 2 line 2 (C_local += SYRK(A_recv)), with X the running sum and Y one more
+ * panel product.  The structure of Z is the union of the two structures; an entry stored in both
+ * gets x + y (one rounded addition in the dtype; I32 wraps), an entry stored in one keeps its
+ * value bit for bit.  Rows of Z are ascending in column.  Z must not alias X or Y.
+ *
+ * Three-step use:
+ *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for m.
+ *   2. d_z_colidx == NULL: writes d_z_rowptr[m + 1] and *nnz_out (synchronises).
+ *   3. all pointers set: fills d_z_colidx / d_z_vals using the d_z_rowptr of step 2.  Asynchronous.
+ * All pointers are device pointers except nnz_out and workspace_bytes (host).
+ * nnz_x = d_x_rowptr[m], nnz_y = d_y_rowptr[m] (they only steer how many lanes share a row).
+ * Errors: INVALID_ARG, WORKSPACE, BAD_CSR (a row of X or Y not strictly ascending), CUDA.
+ */
+spsyrk_status_t spsyrk_accumulate(int64_t m, spsyrk_dtype_t dtype,
+                                  int64_t nnz_x, const int64_t *d_x_rowptr, const int32_t *d_x_colidx, const void *d_x_vals,
+                                  int64_t nnz_y, const int64_t *d_y_rowptr, const int32_t *d_y_colidx, const void *d_y_vals,
+                                  int64_t *d_z_rowptr, int32_t *d_z_colidx, void *d_z_vals,
+                                  int64_t *nnz_out,
+                                  void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
+
+/*
  * spsyrk_symv - y = C x from the stored lower triangle alone,
  *     C x = C_L x + (x^T C_L)^T - D x        (Section V-F, Eq. 1: the triangular output is consumed
  * directly, C_L^T is never formed and the diagonal is counted once).  C_L is any lower-triangular

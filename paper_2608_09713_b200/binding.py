@@ -41,6 +41,8 @@ _lib.spsyrk_plan_set_block.restype = _int
 _lib.spsyrk_symbolic.argtypes = [_vp, _vp, _i64p, _vp]
 _lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
+_lib.spsyrk_column_panel.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
+_lib.spsyrk_accumulate.argtypes = [_i64, _int, _i64, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_mirror_rowptr_noalloc.argtypes = [_i64, _vp, _vp, _vp, _i64p, _vp]
 _lib.spsyrk_mirror_rowptr_noalloc.restype = _int
 _lib.spsyrk_symv.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -60,7 +62,8 @@ _lib.spsyrk_launch_count.restype = ctypes.c_int64
 for _name in ("spsyrk_plan_enable_timing", "spsyrk_plan_timings"):
     getattr(_lib, _name).restype = _int
 for _name in ("spsyrk_plan", "spsyrk_plan_set_rows", "spsyrk_symbolic", "spsyrk_numeric", "spsyrk_mirror",
-              "spsyrk_jaccard", "spsyrk_plan_stats", "spsyrk_plan_buffers", "spsyrk_host_tril"):
+              "spsyrk_jaccard", "spsyrk_plan_stats", "spsyrk_plan_buffers", "spsyrk_host_tril", "spsyrk_column_panel",
+              "spsyrk_accumulate"):
     getattr(_lib, _name).restype = _int
 
 
@@ -256,6 +259,52 @@ def spsyrk_mirror(m, l_rowptr, l_colidx, l_vals, stream=None, workspace=None, ou
     _check(_lib.spsyrk_mirror(m, nnz_l, code, _p(l_rowptr), _p(l_colidx), _p(l_vals), _p(f_rowptr), _p(f_colidx),
                               _p(f_vals), ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_mirror(fill)")
     return f_rowptr, f_colidx[:nnz.value], f_vals[:nnz.value]
+
+
+def spsyrk_column_panel(m, rowptr, colidx, vals, k0, k1, stream=None, workspace=None):
+    """Returns (p_rowptr, p_colidx, p_vals) of A(:, [k0, k1)), column ids unchanged."""
+    _dev_check(rowptr, colidx, vals)
+    nnz, code, dev = colidx.numel(), _DTYPE_CODE[vals.dtype], rowptr.device
+    sz = ctypes.c_size_t(0)
+    _check(_lib.spsyrk_column_panel(m, nnz, code, None, None, None, k0, k1, None, None, None, None, None,
+                                    ctypes.byref(sz), None), "spsyrk_column_panel(size query)")
+    ws = workspace if workspace is not None else _workspace(sz.value, dev)
+    assert ws.numel() >= sz.value
+    sz = ctypes.c_size_t(ws.numel())
+    p_rowptr = torch.empty(m + 1, dtype=torch.int64, device=dev)
+    out_nnz = ctypes.c_int64(0)
+    st = _stream(stream)
+    _check(_lib.spsyrk_column_panel(m, nnz, code, _p(rowptr), _p(colidx), _p(vals), k0, k1, _p(p_rowptr), None, None,
+                                    ctypes.byref(out_nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_column_panel(sizes)")
+    p_colidx = torch.empty(max(out_nnz.value, 1), dtype=torch.int32, device=dev)
+    p_vals = torch.empty(max(out_nnz.value, 1), dtype=vals.dtype, device=dev)
+    _check(_lib.spsyrk_column_panel(m, nnz, code, _p(rowptr), _p(colidx), _p(vals), k0, k1, _p(p_rowptr), _p(p_colidx),
+                                    _p(p_vals), ctypes.byref(out_nnz), _p(ws), ctypes.byref(sz), st), "spsyrk_column_panel(fill)")
+    return p_rowptr, p_colidx[:out_nnz.value], p_vals[:out_nnz.value]
+
+
+def spsyrk_accumulate(m, x_rowptr, x_colidx, x_vals, y_rowptr, y_colidx, y_vals, stream=None, workspace=None):
+    """Returns (z_rowptr, z_colidx, z_vals) of Z = X + Y (union structure, x + y on shared entries)."""
+    _dev_check(x_rowptr, x_colidx, x_vals, y_rowptr, y_colidx, y_vals)
+    assert x_vals.dtype == y_vals.dtype
+    nx, ny, code, dev = x_colidx.numel(), y_colidx.numel(), _DTYPE_CODE[x_vals.dtype], x_rowptr.device
+    sz = ctypes.c_size_t(0)
+    _check(_lib.spsyrk_accumulate(m, code, nx, None, None, None, ny, None, None, None, None, None, None, None, None,
+                                  ctypes.byref(sz), None), "spsyrk_accumulate(size query)")
+    ws = workspace if workspace is not None else _workspace(sz.value, dev)
+    assert ws.numel() >= sz.value
+    sz = ctypes.c_size_t(ws.numel())
+    z_rowptr = torch.empty(m + 1, dtype=torch.int64, device=dev)
+    nnz = ctypes.c_int64(0)
+    st = _stream(stream)
+    args = (m, code, nx, _p(x_rowptr), _p(x_colidx), _p(x_vals), ny, _p(y_rowptr), _p(y_colidx), _p(y_vals), _p(z_rowptr))
+    _check(_lib.spsyrk_accumulate(*args, None, None, ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st),
+           "spsyrk_accumulate(sizes)")
+    z_colidx = torch.empty(max(nnz.value, 1), dtype=torch.int32, device=dev)
+    z_vals = torch.empty(max(nnz.value, 1), dtype=x_vals.dtype, device=dev)
+    _check(_lib.spsyrk_accumulate(*args, _p(z_colidx), _p(z_vals), ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st),
+           "spsyrk_accumulate(fill)")
+    return z_rowptr, z_colidx[:nnz.value], z_vals[:nnz.value]
 
 
 def spsyrk_symv(m, l_rowptr, l_colidx, l_vals, x, y=None, stream=None):

@@ -63,6 +63,14 @@ def test_argument_errors_without_device(lib):
     assert sz.value > 0
     assert lib.spsyrk_mirror(i64(-1), i64(30), 0, None, None, None, None, None, None, None, None, ctypes.byref(sz), None) == 1
     assert lib.spsyrk_jaccard(i64(10), i64(5), i64(6), None, None, None, None, None, None) == 1
+    panel = lambda m, k0, k1: lib.spsyrk_column_panel(i64(m), i64(30), 0, None, None, None, i64(k0), i64(k1), None, None, None,
+                                                      None, None, ctypes.byref(sz), None)
+    assert panel(10, 0, 5) == 0 and sz.value > 0
+    assert panel(10, 5, 4) == 1 and panel(-1, 0, 5) == 1
+    acc = lambda m, dt: lib.spsyrk_accumulate(i64(m), dt, i64(30), None, None, None, i64(20), None, None, None, None, None,
+                                              None, None, None, ctypes.byref(sz), None)
+    assert acc(10, 0) == 0 and sz.value > 0
+    assert acc(-1, 0) == 1 and acc(10, 7) == 1
 
 
 def test_binding_mirrors_the_header():

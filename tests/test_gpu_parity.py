@@ -343,3 +343,102 @@ def test_symv(B, idx):
     exp, scale = oracle.symv(a.m, rp.cpu().numpy(), ci.cpu().numpy(), cv.cpu().numpy().astype(np.float64), x.astype(np.float64))
     tol = 1e-12 if a.vals.dtype == np.float64 else 2e-5
     assert np.all(np.abs(y.astype(np.float64) - exp) <= tol * (scale + 1e-300))
+
+
+# ------------------------------------------- accumulating form over column panels (Section III-A, Algorithm 2)
+def _np(*ts):
+    return [t.cpu().numpy() for t in ts]
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_column_panel(B, idx):
+    a = W.small(idx)
+    d = dev(a)
+    for k0, k1 in [(0, a.n), (0, a.n // 3), (a.n // 3, a.n // 3), (a.n // 3, a.n - 1), (a.n - 1, a.n), (a.n, a.n + 7)]:
+        pr, pc, pv = _np(*B.spsyrk_column_panel(a.m, *d, k0, k1))
+        er, ec, ev = oracle.column_panel(a.m, a.rowptr, a.colidx, a.vals, k0, k1)
+        assert np.array_equal(pr, er) and np.array_equal(pc, ec)
+        assert np.array_equal(pv.astype(np.float64), ev)       # values are copied bit for bit
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("npanels", [2, 5])
+def test_accumulate_panels(B, idx, npanels):
+    """C_L = sum over panels of tril(A_s A_s^T): every step against the oracle's sum of the same operands
+    (bit-exact, one rounded addition per shared entry), the end against the unsplit product."""
+    a = W.small(idx)
+    d = dev(a)
+    edges = np.linspace(0, a.n, npanels + 1).astype(np.int64)
+    acc = None
+    for s in range(npanels):
+        p = B.spsyrk_column_panel(a.m, *d, int(edges[s]), int(edges[s + 1]))
+        t_rowptr, t_colidx, t_vals, _ = B.tril_syrk(a.m, a.n, *p)
+        if acc is None:
+            acc = (t_rowptr, t_colidx, t_vals)
+            continue
+        z = B.spsyrk_accumulate(a.m, *acc, t_rowptr, t_colidx, t_vals)
+        xr, xc, xv, yr, yc, yv = _np(*acc, t_rowptr, t_colidx, t_vals)
+        er, ec, ev = oracle.add(a.m, xr, xc, xv.astype(np.float64), yr, yc, yv.astype(np.float64))
+        zr, zc, zv = _np(*z)
+        assert np.array_equal(zr, er) and np.array_equal(zc, ec)
+        if a.vals.dtype == np.float32:
+            assert np.array_equal(zv, ev.astype(np.float32))   # the double sum of two floats rounds to the float sum
+        else:
+            assert np.array_equal(zv.astype(np.float64), ev)
+        acc = z
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL)
+    zr, zc, zv = _np(*acc)
+    assert np.array_equal(zr, ref.rowptr) and np.array_equal(zc, ref.colidx)   # union of panel structures = structure of the whole
+    check_values(zv, ref, a.vals.dtype)
+
+
+def test_accumulate_edge_cases(B):
+    dev0 = torch.device("cuda")
+    def csr(m, rows):
+        rp = np.zeros(m + 1, dtype=np.int64)
+        ci, va = [], []
+        for i, r in enumerate(rows):
+            rp[i + 1] = rp[i] + len(r)
+            ci += [c for c, _ in r]
+            va += [v for _, v in r]
+        return (torch.from_numpy(rp).to(dev0), torch.tensor(ci, dtype=torch.int32, device=dev0),
+                torch.tensor(va, dtype=torch.float64, device=dev0))
+    # empty + empty, empty + something, cancellation keeps the entry, disjoint and identical rows
+    x = csr(5, [[], [(0, 1.0), (3, 2.0)], [(1, 1.5)], [(0, 1.0), (1, 1.0), (2, 1.0)], []])
+    y = csr(5, [[], [], [(1, -1.5)], [(0, 2.0), (1, 3.0), (2, 4.0)], [(4, 9.0)]])
+    zr, zc, zv = _np(*B.spsyrk_accumulate(5, *x, *y))
+    assert zr.tolist() == [0, 0, 2, 3, 6, 7]
+    assert zc.tolist() == [0, 3, 1, 0, 1, 2, 4]
+    assert zv.tolist() == [1.0, 2.0, 0.0, 3.0, 4.0, 5.0, 9.0]
+    e = csr(5, [[], [], [], [], []])
+    zr, zc, zv = _np(*B.spsyrk_accumulate(5, *e, *e))
+    assert zr.tolist() == [0] * 6 and zc.size == 0
+    # m = 0
+    z0 = csr(0, [])
+    assert B.spsyrk_accumulate(0, *z0, *z0)[0].cpu().tolist() == [0]
+    # a row that is not ascending is refused
+    bad = csr(2, [[(3, 1.0), (1, 1.0)], []])
+    ok = csr(2, [[(1, 1.0)], []])
+    for args in ((bad, ok), (ok, bad)):
+        with pytest.raises(B.SpsyrkError) as ei:
+            B.spsyrk_accumulate(2, *args[0], *args[1])
+        assert ei.value.status == 2
+
+
+def test_accumulate_long_rows(B):
+    """Rows much longer than a group of lanes, with many shared entries (the running match count
+    crosses many 32-entry steps), int32 values."""
+    rng = np.random.default_rng(11)
+    m, n = 37, 20000
+    def rand_csr(density):
+        mask = rng.random((m, n)) < density
+        mask[5] = False
+        rp = np.zeros(m + 1, dtype=np.int64)
+        np.cumsum(mask.sum(axis=1), out=rp[1:])
+        rr, cc = np.nonzero(mask)
+        return rp, cc.astype(np.int32), rng.integers(-5, 6, size=cc.size).astype(np.int32)
+    x, y = rand_csr(0.3), rand_csr(0.4)
+    z = B.spsyrk_accumulate(m, *[torch.from_numpy(t).cuda() for t in x], *[torch.from_numpy(t).cuda() for t in y])
+    er, ec, ev = oracle.add(m, x[0], x[1], x[2].astype(np.float64), y[0], y[1], y[2].astype(np.float64))
+    zr, zc, zv = _np(*z)
+    assert np.array_equal(zr, er) and np.array_equal(zc, ec) and np.array_equal(zv, oracle.to_int32(ev))
