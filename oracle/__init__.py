@@ -49,6 +49,8 @@ def _load():
         lib.oracle_symv.argtypes = [i64, p, p, p, p, p, p]
         lib.oracle_column_panel.argtypes = [i64, p, p, p, i64, i64, p, p, p]
         lib.oracle_add.argtypes = [i64, p, p, p, p, p, p, p, p, p]
+        lib.oracle_permute.argtypes = [i64, i64, p, p, p, p, p, p, p, p]
+        lib.oracle_partition.argtypes = [i64, p, i64, p]
         lib.oracle_symv.restype = ctypes.c_int
         for f in (lib.oracle_transpose, lib.oracle_syrk_rows, lib.oracle_mirror, lib.oracle_jaccard):
             f.restype = ctypes.c_int
@@ -206,3 +208,30 @@ def add(m, x_rowptr, x_colidx, x_vals, y_rowptr, y_colidx, y_vals):
     rc = lib.oracle_add(*args, _ptr(z_rowptr), _ptr(z_colidx), _ptr(z_vals))
     assert rc == 0
     return z_rowptr, z_colidx[:nnz], z_vals[:nnz]
+
+
+def permute(m, n, rowptr, colidx, vals, rperm, cperm=None):
+    """B with row i of A at row rperm[i] and column k at column cperm[k] (None: columns stay);
+    rows of B ascending in column.  Returns (rowptr, colidx, vals float64)."""
+    lib = _load()
+    rowptr, colidx, vals = _c(rowptr, np.int64), _c(colidx, np.int32), _c(vals, np.float64)
+    rperm = _c(rperm, np.int32)
+    cperm = None if cperm is None else _c(cperm, np.int32)
+    nnz = int(rowptr[m])
+    b_rowptr = np.empty(m + 1, dtype=np.int64)
+    b_colidx = np.empty(max(nnz, 1), dtype=np.int32)
+    b_vals = np.empty(max(nnz, 1), dtype=np.float64)
+    rc = lib.oracle_permute(m, n, _ptr(rowptr), _ptr(colidx), _ptr(vals), _ptr(rperm), _ptr(cperm),
+                            _ptr(b_rowptr), _ptr(b_colidx), _ptr(b_vals))
+    assert rc == 0, "not a permutation"
+    return b_rowptr, b_colidx[:nnz], b_vals[:nnz]
+
+
+def partition(work, parts) -> np.ndarray:
+    """Row bounds (parts + 1 int64) of contiguous ranges with near-equal sums of `work`."""
+    lib = _load()
+    work = _c(work, np.int64)
+    bounds = np.empty(parts + 1, dtype=np.int64)
+    rc = lib.oracle_partition(work.size, _ptr(work), parts, _ptr(bounds))
+    assert rc == 0
+    return bounds

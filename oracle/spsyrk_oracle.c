@@ -259,3 +259,63 @@ int oracle_add(int64_t m, const int64_t *x_rowptr, const int32_t *x_colidx, cons
     if (!z_colidx) z_rowptr[m] = o;
     return 0;
 }
+
+/* B = P A Q^T for permutations given as maps: row i of A becomes row rperm[i] of B and column k
+ * becomes column cperm[k] (cperm == NULL: columns stay).  With a square A and cperm == rperm this
+ * is the symmetric random permutation that restores load balance (Section III-A; the load
+ * balance study of Section V).  Rows of B are ascending in column again.  b_rowptr[m+1],
+ * b_colidx[nnz], b_vals[nnz].  Returns 0, or -2 if a map is not a permutation. */
+int oracle_permute(int64_t m, int64_t n, const int64_t *rowptr, const int32_t *colidx, const double *vals,
+                   const int32_t *rperm, const int32_t *cperm,
+                   int64_t *b_rowptr, int32_t *b_colidx, double *b_vals)
+{
+    char *seen = (char *)calloc((size_t)((m > n ? m : n) + 1), 1);
+    if (!seen) return -1;
+    for (int64_t i = 0; i < m; ++i) {
+        if (rperm[i] < 0 || rperm[i] >= m || seen[rperm[i]]) { free(seen); return -2; }
+        seen[rperm[i]] = 1;
+    }
+    if (cperm) {
+        memset(seen, 0, (size_t)((m > n ? m : n) + 1));
+        for (int64_t k = 0; k < n; ++k) {
+            if (cperm[k] < 0 || cperm[k] >= n || seen[cperm[k]]) { free(seen); return -2; }
+            seen[cperm[k]] = 1;
+        }
+    }
+    free(seen);
+    memset(b_rowptr, 0, (size_t)(m + 1) * sizeof(int64_t));
+    for (int64_t i = 0; i < m; ++i) b_rowptr[rperm[i] + 1] = rowptr[i + 1] - rowptr[i];
+    for (int64_t i = 0; i < m; ++i) b_rowptr[i + 1] += b_rowptr[i];
+    for (int64_t i = 0; i < m; ++i) {
+        int64_t o = b_rowptr[rperm[i]], len = 0;
+        for (int64_t p = rowptr[i]; p < rowptr[i + 1]; ++p) {
+            int32_t c = cperm ? cperm[colidx[p]] : colidx[p];
+            double v = vals[p];
+            int64_t q = o + len;   /* insertion into the ascending destination row */
+            while (q > o && b_colidx[q - 1] > c) { b_colidx[q] = b_colidx[q - 1]; b_vals[q] = b_vals[q - 1]; --q; }
+            b_colidx[q] = c;
+            b_vals[q] = v;
+            ++len;
+        }
+    }
+    return 0;
+}
+
+/* Contiguous row ranges of near-equal work for a 1-D distribution of the output rows (the work
+ * of the lower triangle grows with the row index, so equal row counts are not equal work):
+ * bounds[0] = 0, bounds[parts] = rows, and bounds[p] is the smallest r whose work prefix
+ * sum_{i<r} work[i] reaches p/parts of the total.  Returns 0. */
+int oracle_partition(int64_t rows, const int64_t *work, int64_t parts, int64_t *bounds)
+{
+    long double total = 0;
+    for (int64_t i = 0; i < rows; ++i) total += (long double)work[i];
+    int64_t r = 0;
+    long double prefix = 0;   /* exact: integer values far below 2^64 */
+    bounds[0] = 0;
+    for (int64_t p = 1; p < parts; ++p) {
+        while (r < rows && prefix * (long double)parts < (long double)p * total) { prefix += (long double)work[r]; ++r; }
+        bounds[p] = r;
+    }
+    bounds[parts] = rows;
+    return 0;
+}

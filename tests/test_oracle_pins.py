@@ -488,3 +488,86 @@ def test_panel_products_sum_to_the_whole(small_case, npanels):
         assert np.array_equal(zv, tril.vals)
     else:
         assert np.all(np.abs(zv - tril.vals) <= 1e-13 * tril.absvals)
+
+
+# ------------------------------------- symmetric permutation and row ranges of equal work
+@pytest.mark.parametrize("seed", range(3))
+def test_permute_dense_definition(seed):
+    """Pin: B[rperm[i], cperm[k]] = A[i, k] evaluated on dense arrays, stored zeros kept."""
+    rng = np.random.default_rng(300 + seed)
+    m, n = 11, 14
+    d = rng.integers(-3, 4, size=(m, n)).astype(np.float64)
+    st = rng.random((m, n)) < 0.35
+    st[4] = False
+    a = csr_from_dense(d, st)
+    rp, cp = rng.permutation(m).astype(np.int32), rng.permutation(n).astype(np.int32)
+    for cperm in (cp, None):
+        br, bc, bv = oracle.permute(m, n, a.rowptr, a.colidx, a.vals, rp, cperm)
+        eb, es = np.zeros((m, n)), np.zeros((m, n), dtype=bool)
+        cmap = np.arange(n) if cperm is None else cperm
+        for i in range(m):
+            for k in range(n):
+                if st[i, k]:
+                    eb[rp[i], cmap[k]] = d[i, k]
+                    es[rp[i], cmap[k]] = True
+        e = csr_from_dense(eb, es)
+        assert np.array_equal(br, e.rowptr) and np.array_equal(bc, e.colidx) and np.array_equal(bv, e.vals)
+
+
+def test_permute_matches_scipy_indexing(small_case):
+    """Pin: scipy fancy indexing (third party): B = A[inv_r][:, inv_c]."""
+    cfg, a, _, _ = small_case
+    rng = np.random.default_rng(cfg)
+    rp, cp = rng.permutation(a.m).astype(np.int32), rng.permutation(a.n).astype(np.int32)
+    s = sp.csr_matrix((a.vals.astype(np.float64), a.colidx, a.rowptr), shape=(a.m, a.n))
+    inv_r, inv_c = np.argsort(rp), np.argsort(cp)
+    ref = s[inv_r][:, inv_c].tocsr()
+    ref.sort_indices()
+    br, bc, bv = oracle.permute(a.m, a.n, a.rowptr, a.colidx, a.vals, rp, cp)
+    assert np.array_equal(br, ref.indptr) and np.array_equal(bc, ref.indices) and np.array_equal(bv, ref.data)
+
+
+def test_permuted_product_is_permuted_product():
+    """Pin: (P A)(P A)^T = P (A A^T) P^T, so the full product of the permuted matrix is the
+    symmetric permutation of the full product; a column permutation changes nothing but the order
+    of the additions (integer values: exact)."""
+    a = W.small(4)
+    rng = np.random.default_rng(9)
+    rp, cp = rng.permutation(a.m).astype(np.int32), rng.permutation(a.n).astype(np.int32)
+    full = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.FULL)
+    b = oracle.permute(a.m, a.n, a.rowptr, a.colidx, a.vals, rp, cp)
+    fb = oracle.syrk(a.m, a.n, *b, oracle.FULL)
+    pr, pc, pv = oracle.permute(a.m, a.m, full.rowptr, full.colidx, full.vals, rp, rp)
+    assert np.array_equal(fb.rowptr, pr) and np.array_equal(fb.colidx, pc) and np.array_equal(fb.vals, pv)
+
+
+def test_permute_rejects_non_permutations():
+    a = W.small(1)
+    bad = np.zeros(a.m, dtype=np.int32)
+    with pytest.raises(AssertionError):
+        oracle.permute(a.m, a.n, a.rowptr, a.colidx, a.vals, bad)
+
+
+def test_partition_definition_and_invariants(small_case):
+    """Pin: the definition by brute force (exact integer arithmetic in Python), plus what any such
+    split must satisfy: monotone bounds covering all rows, and no part heavier than its share by
+    more than one row's work."""
+    _, a, _, tril = small_case
+    work = tril.work
+    total = int(work.sum())
+    prefix = np.concatenate([[0], np.cumsum(work)])
+    for parts in (1, 2, 3, 8, 64):
+        b = oracle.partition(work, parts)
+        assert b[0] == 0 and b[parts] == a.m and np.all(np.diff(b) >= 0)
+        for p in range(1, parts):
+            r = next(r for r in range(a.m + 1) if int(prefix[r]) * parts >= p * total)
+            assert b[p] == r
+        share = [int(prefix[b[p + 1]] - prefix[b[p]]) for p in range(parts)]
+        assert sum(share) == total
+        assert max(share) <= total / parts + int(work.max()) + 1
+
+
+def test_partition_degenerate():
+    assert oracle.partition(np.zeros(5, dtype=np.int64), 3).tolist() == [0, 0, 0, 5]
+    assert oracle.partition(np.zeros(0, dtype=np.int64), 2).tolist() == [0, 0, 0]
+    assert oracle.partition(np.array([7], dtype=np.int64), 4).tolist() == [0, 1, 1, 1, 1]
