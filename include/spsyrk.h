@@ -195,6 +195,37 @@ spsyrk_status_t spsyrk_accumulate(int64_t m, spsyrk_dtype_t dtype,
                                   void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
 
 /*
+ * spsyrk_permute - B = P A Q^T as canonical CSR: row i of A becomes row d_rperm[i] of B and column k
+ * becomes column d_cperm[k] (d_cperm == NULL: columns stay).  With a square A and the same map
+ * for rows and columns this is the symmetric random permutation that restores load balance
+ * (Section III-A; the load-balance study of Section V).  Rows of B are ascending in column.
+ *
+ * Two-step use:
+ *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for (m, n, nnz, dtype).
+ *   2. all pointers set: writes d_b_rowptr[m + 1], d_b_colidx[nnz], d_b_vals[nnz] (synchronises).
+ * All pointers are device pointers except workspace_bytes (host); d_rperm has m entries, d_cperm n;
+ * d_vals must be 16-byte aligned; B must not alias A.  Errors: INVALID_ARG (also: a map that is
+ * not a permutation), WORKSPACE, OVERFLOW, BAD_CSR (row pointers or column ids out of range), CUDA.
+ */
+spsyrk_status_t spsyrk_permute(int64_t m, int64_t n, int64_t nnz, spsyrk_dtype_t dtype,
+                               const int64_t *d_rowptr, const int32_t *d_colidx, const void *d_vals,
+                               const int32_t *d_rperm, const int32_t *d_cperm,
+                               int64_t *d_b_rowptr, int32_t *d_b_colidx, void *d_b_vals,
+                               void *d_workspace, size_t *workspace_bytes, void *cuda_stream);
+
+/*
+ * spsyrk_plan_partition - contiguous ranges of the plan's output rows with near-equal work, for a
+ * 1-D distribution of the rows over `parts` workers (the work of the lower triangle grows with
+ * the row index, so equal row counts are not equal work; Section III-A asks for balanced work).
+ * bounds (HOST, parts + 1 entries) receives absolute row ids: bounds[0] = row_begin,
+ * bounds[parts] = row_end, and bounds[p] is the first row at which the prefix sum of the per-row
+ * work estimate reaches p/parts of the total.  Worker p then calls spsyrk_plan_set_rows with
+ * [bounds[p], bounds[p + 1]).  1 <= parts <= 65536.  Synchronises.
+ * Errors: INVALID_ARG, OVERFLOW (total work x parts does not fit 63 bits), CUDA.
+ */
+spsyrk_status_t spsyrk_plan_partition(spsyrk_plan_t plan, int64_t parts, int64_t *bounds, void *cuda_stream);
+
+/*
  * spsyrk_symv - y = C x from the stored lower triangle alone,
  *     C x = C_L x + (x^T C_L)^T - D x        (Section V-F, Eq. 1: the triangular output is consumed
  * directly, C_L^T is never formed and the diagonal is counted once).  C_L is any lower-triangular

@@ -43,6 +43,8 @@ _lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_column_panel.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_accumulate.argtypes = [_i64, _int, _i64, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
+_lib.spsyrk_permute.argtypes = [_i64, _i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _szp, _vp]
+_lib.spsyrk_plan_partition.argtypes = [_vp, _i64, _i64p, _vp]
 _lib.spsyrk_mirror_rowptr_noalloc.argtypes = [_i64, _vp, _vp, _vp, _i64p, _vp]
 _lib.spsyrk_mirror_rowptr_noalloc.restype = _int
 _lib.spsyrk_symv.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -63,7 +65,7 @@ for _name in ("spsyrk_plan_enable_timing", "spsyrk_plan_timings"):
     getattr(_lib, _name).restype = _int
 for _name in ("spsyrk_plan", "spsyrk_plan_set_rows", "spsyrk_symbolic", "spsyrk_numeric", "spsyrk_mirror",
               "spsyrk_jaccard", "spsyrk_plan_stats", "spsyrk_plan_buffers", "spsyrk_host_tril", "spsyrk_column_panel",
-              "spsyrk_accumulate"):
+              "spsyrk_accumulate", "spsyrk_permute", "spsyrk_plan_partition"):
     getattr(_lib, _name).restype = _int
 
 
@@ -305,6 +307,35 @@ def spsyrk_accumulate(m, x_rowptr, x_colidx, x_vals, y_rowptr, y_colidx, y_vals,
     _check(_lib.spsyrk_accumulate(*args, _p(z_colidx), _p(z_vals), ctypes.byref(nnz), _p(ws), ctypes.byref(sz), st),
            "spsyrk_accumulate(fill)")
     return z_rowptr, z_colidx[:nnz.value], z_vals[:nnz.value]
+
+
+def spsyrk_permute(m, n, rowptr, colidx, vals, rperm, cperm=None, stream=None, workspace=None):
+    """Returns (b_rowptr, b_colidx, b_vals): row i of A at row rperm[i], column k at column cperm[k]
+    (None: columns stay); rperm / cperm are int32 CUDA tensors."""
+    _dev_check(rowptr, colidx, vals, rperm, cperm)
+    assert rperm.dtype == torch.int32 and rperm.numel() == m
+    assert cperm is None or (cperm.dtype == torch.int32 and cperm.numel() == n)
+    nnz, code, dev = colidx.numel(), _DTYPE_CODE[vals.dtype], rowptr.device
+    sz = ctypes.c_size_t(0)
+    _check(_lib.spsyrk_permute(m, n, nnz, code, None, None, None, None, None, None, None, None, None, ctypes.byref(sz), None),
+           "spsyrk_permute(size query)")
+    ws = workspace if workspace is not None else _workspace(sz.value, dev)
+    assert ws.numel() >= sz.value
+    sz = ctypes.c_size_t(ws.numel())
+    b_rowptr = torch.empty(m + 1, dtype=torch.int64, device=dev)
+    b_colidx = torch.empty(max(nnz, 1), dtype=torch.int32, device=dev)
+    b_vals = torch.empty(max(nnz, 1), dtype=vals.dtype, device=dev)
+    _check(_lib.spsyrk_permute(m, n, nnz, code, _p(rowptr), _p(colidx), _p(vals), _p(rperm), _p(cperm), _p(b_rowptr),
+                               _p(b_colidx), _p(b_vals), _p(ws), ctypes.byref(sz), _stream(stream)), "spsyrk_permute")
+    return b_rowptr, b_colidx[:nnz], b_vals[:nnz]
+
+
+def spsyrk_plan_partition(plan, parts, stream=None):
+    """Row bounds (list of parts + 1 absolute row ids) of contiguous ranges of the plan's rows with
+    near-equal work; worker p takes [bounds[p], bounds[p + 1])."""
+    out = (ctypes.c_int64 * (parts + 1))()
+    _check(_lib.spsyrk_plan_partition(plan._h, parts, out, _stream(stream)), "spsyrk_plan_partition")
+    return list(out)
 
 
 def spsyrk_symv(m, l_rowptr, l_colidx, l_vals, x, y=None, stream=None):

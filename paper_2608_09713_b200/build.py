@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspsyrk.so")
-SOURCES = ["api.cu", "mirror.cu", "jaccard.cu", "symv.cu", "accumulate.cu", "host.cu"]
+SOURCES = ["api.cu", "mirror.cu", "jaccard.cu", "symv.cu", "accumulate.cu", "permute.cu", "host.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",
               "-Wno-deprecated-gpu-targets"]

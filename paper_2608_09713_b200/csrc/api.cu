@@ -26,6 +26,7 @@ constexpr int TRANSPOSE_RADIX_BITS = 8;
 constexpr size_t LARGE_SMEM_BUDGET = 200 * 1024;
 constexpr int GLOBAL_ACC_CTAS = 160;  // upper bound of the persistent heavy-row grid (one CTA per SM)
 constexpr uint32_t BLOCK_ACC_SLOTS = 4096;
+constexpr int64_t MAX_PARTS = 65536;
 
 size_t dtype_size(spsyrk_dtype_t t) { return t == SPSYRK_F64 ? 8 : 4; }
 
@@ -75,6 +76,8 @@ struct spsyrk_plan_s {
     uint32_t* row_counter;  // row dispenser of the persistent heavy-row kernel
     double* gacc;           // its global accumulator slices (GLOBAL_ACC_CTAS x gslots, 8 bytes per slot)
     uint32_t gslots;
+    int64_t* work_prefix;  // rows + 1: exclusive prefix sums of the per-row work (spsyrk_plan_partition)
+    int64_t* part_bounds;  // MAX_PARTS + 1
     // host facts
     int64_t class_start[NCLASS + 1];
     int64_t work_total;
@@ -120,11 +123,14 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     auto work_total_dev = c.take<unsigned long long>(1);
     auto err = c.take<uint32_t>(1);
     auto row_counter = c.take<uint32_t>(1);
+    auto work_prefix = c.take<int64_t>(items + 1);
+    auto part_bounds = c.take<int64_t>(MAX_PARTS + 1);
     // one global accumulator slice per persistent CTA of the heavy-row numeric kernel
     const uint32_t gslots = pow2_at_least((uint64_t)std::max<int64_t>(m, 1), 1024u, ROW_CHUNK_BITS_MAX_NUMERIC);
     auto gacc = c.take<double>((size_t)GLOBAL_ACC_CTAS * gslots);
     if (pl) {
         pl->row_counter = row_counter; pl->gacc = gacc; pl->gslots = gslots;
+        pl->work_prefix = work_prefix; pl->part_bounds = part_bounds;
         pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.desc = desc;
         pl->dev.work = work; pl->dev.err = err;
         pl->desc_full = desc; pl->desc_blk = desc_blk;
@@ -297,6 +303,21 @@ void launch_numeric_warp_all(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t
     mark(pl, pl->ev_num, 6, st);
 }
 
+// bounds[p] = r0 + the smallest r in [0, rows] with prefix[r] * parts >= p * prefix[rows]
+__global__ void partition_kernel(const int64_t* __restrict__ prefix, int64_t rows, int64_t parts, int64_t r0,
+                                 int64_t* __restrict__ bounds) {
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p > parts) return;
+    if (p == parts) { bounds[p] = r0 + rows; return; }
+    const int64_t target = p * prefix[rows];
+    int64_t lo = 0, hi = rows;  // prefix is non-decreasing; prefix[rows] * parts >= target always
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (prefix[mid] * parts >= target) hi = mid; else lo = mid + 1;
+    }
+    bounds[p] = r0 + lo;
+}
+
 uint32_t row_chunk_bits(const spsyrk_plan_s* pl, uint32_t cap) {
     const uint64_t umax = pl->dev.mode == SPSYRK_TRIL ? (uint64_t)pl->dev.r1 : (uint64_t)pl->dev.m;
     return pow2_at_least(umax, 1024u, cap);
@@ -460,6 +481,21 @@ spsyrk_status_t spsyrk_plan_set_block(spsyrk_plan_t plan, int64_t row_begin, int
 spsyrk_status_t spsyrk_plan_set_rows(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end, void* cuda_stream) {
     if (!plan) return SPSYRK_ERR_INVALID_ARG;
     return spsyrk_plan_set_block(plan, row_begin, row_end, 0, plan->dev.m, cuda_stream);
+}
+
+spsyrk_status_t spsyrk_plan_partition(spsyrk_plan_t plan, int64_t parts, int64_t* bounds, void* cuda_stream) {
+    if (!plan || !bounds || parts < 1 || parts > MAX_PARTS) return SPSYRK_ERR_INVALID_ARG;
+    spsyrk_plan_s* pl = plan;
+    if (pl->work_total > 0 && pl->work_total > INT64_MAX / parts) return SPSYRK_ERR_OVERFLOW;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t rows = pl->dev.r1 - pl->dev.r0;
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<int64_t>(pl->dev.work, rows, pl->work_prefix, pl->partials, st));
+    partition_kernel<<<(unsigned)((parts + 1 + 255) / 256), 256, 0, st>>>(pl->work_prefix, rows, parts, pl->dev.r0, pl->part_bounds);
+    note_launches(1);
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(bounds, pl->part_bounds, (size_t)(parts + 1) * sizeof(int64_t), cudaMemcpyDeviceToHost, st));
+    SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
+    return SPSYRK_OK;
 }
 
 spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t* d_c_rowptr, int64_t* nnz_out, void* cuda_stream) {

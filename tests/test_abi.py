@@ -71,6 +71,11 @@ def test_argument_errors_without_device(lib):
                                               None, None, None, ctypes.byref(sz), None)
     assert acc(10, 0) == 0 and sz.value > 0
     assert acc(-1, 0) == 1 and acc(10, 7) == 1
+    perm = lambda m, n: lib.spsyrk_permute(i64(m), i64(n), i64(30), 0, None, None, None, None, None, None, None, None, None,
+                                           ctypes.byref(sz), None)
+    assert perm(10, 12) == 0 and sz.value > 0
+    assert perm(-1, 12) == 1 and perm(1 << 31, 12) == 4
+    assert lib.spsyrk_plan_partition(None, i64(4), None, None) == 1
 
 
 def test_binding_mirrors_the_header():

@@ -442,3 +442,82 @@ def test_accumulate_long_rows(B):
     er, ec, ev = oracle.add(m, x[0], x[1], x[2].astype(np.float64), y[0], y[1], y[2].astype(np.float64))
     zr, zc, zv = _np(*z)
     assert np.array_equal(zr, er) and np.array_equal(zc, ec) and np.array_equal(zv, oracle.to_int32(ev))
+
+
+# ------------------------------ symmetric permutation and equal-work row ranges (Section III-A, load balance)
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_permute(B, idx):
+    a = W.small(idx)
+    d = dev(a)
+    rng = np.random.default_rng(40 + idx)
+    rp, cp = rng.permutation(a.m).astype(np.int32), rng.permutation(a.n).astype(np.int32)
+    for cperm in (cp, None):
+        got = _np(*B.spsyrk_permute(a.m, a.n, *d, torch.from_numpy(rp).cuda(), None if cperm is None else torch.from_numpy(cperm).cuda()))
+        er, ec, ev = oracle.permute(a.m, a.n, a.rowptr, a.colidx, a.vals, rp, cperm)
+        assert np.array_equal(got[0], er) and np.array_equal(got[1], ec)
+        assert np.array_equal(got[2].astype(np.float64), ev)   # values are moved bit for bit
+
+
+def test_permute_then_product(B):
+    """The product of the symmetrically permuted matrix against the oracle on the same permuted input."""
+    a = W.small(3)
+    rng = np.random.default_rng(5)
+    perm = rng.permutation(a.m).astype(np.int32)
+    pt = torch.from_numpy(perm).cuda()
+    b = B.spsyrk_permute(a.m, a.n, *dev(a), pt, pt)
+    br, bc, bv = _np(*b)
+    pa = W.CSR(a.m, a.n, br, bc, bv)
+    run_and_compare(B, pa, 0)
+
+
+def test_permute_edge_cases(B):
+    a = W.small(1)
+    d = dev(a)
+    ident = torch.arange(a.m, dtype=torch.int32, device="cuda")
+    got = _np(*B.spsyrk_permute(a.m, a.n, *d, ident, torch.arange(a.n, dtype=torch.int32, device="cuda")))
+    assert np.array_equal(got[0], a.rowptr) and np.array_equal(got[1], a.colidx) and np.array_equal(got[2], a.vals)
+    bad = ident.clone()
+    bad[3] = bad[4]
+    with pytest.raises(B.SpsyrkError) as ei:
+        B.spsyrk_permute(a.m, a.n, *d, bad)
+    assert ei.value.status == 1
+    bad = ident.clone()
+    bad[0] = a.m
+    with pytest.raises(B.SpsyrkError):
+        B.spsyrk_permute(a.m, a.n, *d, bad)
+    # no rows, no entries
+    e = (torch.zeros(1, dtype=torch.int64, device="cuda"), torch.zeros(0, dtype=torch.int32, device="cuda"),
+         torch.zeros(0, dtype=torch.float64, device="cuda"))
+    assert B.spsyrk_permute(0, 5, *e, torch.zeros(0, dtype=torch.int32, device="cuda"))[0].cpu().tolist() == [0]
+    z = (torch.zeros(4, dtype=torch.int64, device="cuda"), torch.zeros(0, dtype=torch.int32, device="cuda"),
+         torch.zeros(0, dtype=torch.float64, device="cuda"))
+    assert B.spsyrk_permute(3, 5, *z, torch.tensor([2, 0, 1], dtype=torch.int32, device="cuda"))[0].cpu().tolist() == [0, 0, 0, 0]
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_plan_partition(B, idx):
+    a = W.small(idx)
+    plan = B.spsyrk_plan(a.m, a.n, *dev(a))
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, counts_only=True)
+    for parts in (1, 2, 3, 8, 64):
+        assert B.spsyrk_plan_partition(plan, parts) == oracle.partition(ref.work, parts).tolist()
+    # a row range: bounds are absolute row ids inside it
+    r0, r1 = a.m // 4, a.m - a.m // 3
+    B.spsyrk_plan_set_rows(plan, r0, r1)
+    got = B.spsyrk_plan_partition(plan, 5)
+    assert got == (oracle.partition(ref.work[r0:r1], 5) + r0).tolist()
+    # the ranges tile the product: concatenating the parts gives the whole
+    whole = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, r0, r1)
+    pieces = []
+    for p in range(5):
+        if got[p + 1] > got[p]:
+            B.spsyrk_plan_set_rows(plan, got[p], got[p + 1])
+            rp = torch.empty(got[p + 1] - got[p] + 1, dtype=torch.int64, device="cuda")
+            nnz = B.spsyrk_symbolic(plan, rp)
+            ci = torch.empty(max(nnz, 1), dtype=torch.int32, device="cuda")
+            cv = torch.empty(max(nnz, 1), dtype=torch.from_numpy(a.vals).dtype, device="cuda")
+            B.spsyrk_numeric(plan, rp, ci, cv)
+            pieces.append(ci[:nnz].cpu().numpy())
+    assert np.array_equal(np.concatenate(pieces), whole.colidx)
+    with pytest.raises(B.SpsyrkError):
+        B.spsyrk_plan_partition(plan, 0)
