@@ -185,7 +185,7 @@ def run_ours(args):
     if args.zipf_rows:
         a = W.zipf_binary(args.zipf_rows, 1 << 22, 100, 1.1, W.SEED + 2)
     if args.rmat_scale:
-        a = W.rmat(args.rmat_scale, 16, W.SEED + 3)
+        a = W.rmat(args.rmat_scale, 16, W.SEED + 3, permute=not args.rmat_noperm)
     sv = a.vals.dtype.itemsize
     dname = {np.dtype(np.float64): "f64", np.dtype(np.float32): "f32", np.dtype(np.int32): "i32"}[a.vals.dtype]
     d_rowptr, d_colidx, d_vals = (torch.from_numpy(x).cuda() for x in (a.rowptr, a.colidx, a.vals))
@@ -338,6 +338,48 @@ def run_ours(args):
             sm = float(np.mean(st_[1:]))
             line["symv"] = {"ms": sm, "bytes": int(sb), "gbs": sb / (sm / 1e3) / 1e9, "frac_of_peak": sb / (sm / 1e3) / 1e9 / peak}
             del xv, yv
+        # ---- 1-D row sharding study (load balance): symbolic + numeric time of each of 8 contiguous row ranges,
+        # cut by equal row counts and by equal work (spsyrk_plan_partition); the slowest range is what a
+        # row-distributed run would wait for
+        parts = 8
+        splan = B.spsyrk_plan(a.m, a.n, d_rowptr, d_colidx, d_vals, mode=B.TRIL, workspace=buf["plan_ws"])
+        splits = {"equal_work": B.spsyrk_plan_partition(splan, parts), "equal_rows": [a.m * p // parts for p in range(parts + 1)]}
+        prefix = np.concatenate([[0], np.cumsum(work)])
+        shard = {"parts": parts}
+        for nm, bounds in splits.items():
+            ms_parts = []
+            for p_ in range(parts):
+                r0_, r1_ = int(bounds[p_]), int(bounds[p_ + 1])
+                if r1_ <= r0_:
+                    ms_parts.append(0.0)
+                    continue
+                B.spsyrk_plan_set_rows(splan, r0_, r1_)
+                for it in range(2):
+                    e0 = ev()
+                    B.spsyrk_symbolic(splan, buf["c_rowptr"])
+                    B.spsyrk_numeric(splan, buf["c_rowptr"], buf["c_colidx"], buf["c_vals"])
+                    e1 = ev()
+                    torch.cuda.synchronize()
+                ms_parts.append(e0.elapsed_time(e1))
+            share = np.diff(prefix[np.asarray(bounds)]).astype(np.float64)
+            shard[nm] = {"work_max_over_mean": float(share.max() / max(share.mean(), 1.0)),
+                         "ms_max_over_mean": float(max(ms_parts) / max(np.mean(ms_parts), 1e-9)),
+                         "ms_max": float(max(ms_parts)), "ms_sum": float(sum(ms_parts))}
+        line["row_sharding"] = shard
+        del splan
+        if a.m == a.n and not is_int:
+            # the symmetric random permutation as a device pre-pass (same map for rows and columns)
+            g = torch.Generator(device="cpu").manual_seed(1234)
+            pm = torch.randperm(a.m, generator=g).to(torch.int32).cuda()
+            for it in range(2):
+                torch.cuda.synchronize()
+                e0 = ev()
+                pb = B.spsyrk_permute(a.m, a.n, d_rowptr, d_colidx, d_vals, pm, pm)
+                e1 = ev()
+                torch.cuda.synchronize()
+                del pb
+            line["permute_ms"] = e0.elapsed_time(e1)
+            del pm
         del keep
         buf.pop("f", None); buf.pop("mirror_ws", None)
         torch.cuda.empty_cache()
@@ -458,6 +500,7 @@ def main():
     ap.add_argument("--no-mirror", action="store_true")
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--rmat-noperm", action="store_true", help="with --rmat-scale: skip the random relabelling (load-balance study)")
     ap.add_argument("--skip-extras", action="store_true", help="timed steps only (for profiler runs)")
     ap.add_argument("--zipf-rows", type=int, default=0,
                     help="profiling aid: replace the workload by the binary Zipf recipe with this many rows")
