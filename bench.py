@@ -100,6 +100,17 @@ def max_over_ranks(x: float, device="cpu") -> float:
     return float(t.item())
 
 
+def sum_over_ranks(x: float, device="cpu") -> float:
+    """Sum of a per-rank number over all ranks (row-sharded runs: every rank does a part of one job)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
 def whole_job_rate(units_per_rank: float, world: int, ms_per_step: float) -> float:
     """Replicas: every rank processes `units_per_rank` per step; the job's rate counts all of them."""
     return world * units_per_rank / (ms_per_step / 1e3)
@@ -188,10 +199,35 @@ def run_ours(args):
         a = W.rmat(args.rmat_scale, 16, W.SEED + 3, permute=not args.rmat_noperm)
     sv = a.vals.dtype.itemsize
     dname = {np.dtype(np.float64): "f64", np.dtype(np.float32): "f32", np.dtype(np.int32): "i32"}[a.vals.dtype]
-    d_rowptr, d_colidx, d_vals = (torch.from_numpy(x).cuda() for x in (a.rowptr, a.colidx, a.vals))
     is_int = a.vals.dtype == np.int32
-    do_mirror = not (args.no_mirror or is_int)  # the 1e5 x 1e5 dense mirror of config 2 is not asked for
+    shard = bool(args.shard_rows) and world > 1
+    do_mirror = not (args.no_mirror or is_int or shard)  # the 1e5 x 1e5 dense mirror of config 2 is not asked for
     stream = torch.cuda.current_stream()
+    r0, r1, allgather_ms = 0, a.m, None
+    if shard:
+        # Row-sharded run of ONE product: every rank starts with a slice of A's rows, the slices are
+        # all-gathered over NCCL into each GPU's own memory, then each rank computes a range of output rows
+        # of near-equal work.  No collective follows on the data path.
+        from paper_2608_09713_b200 import sharding as S
+        sb = S.row_slice_bounds(a.m, world)
+        s0, s1 = sb[rank], sb[rank + 1]
+        loc = (torch.from_numpy(a.rowptr[s0:s1 + 1] - a.rowptr[s0]).cuda(), torch.from_numpy(a.colidx[a.rowptr[s0]:a.rowptr[s1]]).cuda(),
+               torch.from_numpy(a.vals[a.rowptr[s0]:a.rowptr[s1]]).cuda())
+        for it in range(2):
+            dist.barrier()
+            torch.cuda.synchronize()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            d_rowptr, d_colidx, d_vals = S.allgather_csr(a.m, *loc)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            allgather_ms = max_over_ranks(e0.elapsed_time(e1), "cuda")
+        del loc
+        p0 = B.spsyrk_plan(a.m, a.n, d_rowptr, d_colidx, d_vals, mode=B.TRIL)
+        r0, r1 = S.rank_rows(B.spsyrk_plan_partition(p0, world), rank)
+        del p0
+    else:
+        d_rowptr, d_colidx, d_vals = (torch.from_numpy(x).cuda() for x in (a.rowptr, a.colidx, a.vals))
 
     def ev():
         e = torch.cuda.Event(enable_timing=True)
@@ -200,7 +236,7 @@ def run_ours(args):
 
     # Device buffers are allocated once (sizes come from an untimed sizing pass) and reused by every
     # step, so that no allocator call sits inside the timed region.
-    sizing = B.tril_syrk(a.m, a.n, d_rowptr, d_colidx, d_vals)
+    sizing = B.tril_syrk(a.m, a.n, d_rowptr, d_colidx, d_vals, row_begin=r0, row_end=r1)
     nnz0 = sizing[1].numel()
     del sizing
     torch.cuda.empty_cache()
@@ -221,6 +257,8 @@ def run_ours(args):
         plan = B.spsyrk_plan(a.m, a.n, d_rowptr, d_colidx, d_vals, mode=B.TRIL, workspace=buf["plan_ws"])
         if timing:
             B.spsyrk_plan_enable_timing(plan)
+        if shard:
+            B.spsyrk_plan_set_rows(plan, *S.rank_rows(B.spsyrk_plan_partition(plan, world), rank))
         marks.append(ev())
         c_rowptr, c_colidx, c_vals = buf["c_rowptr"], buf["c_colidx"], buf["c_vals"]
         nnz = B.spsyrk_symbolic(plan, c_rowptr)
@@ -271,18 +309,29 @@ def run_ours(args):
     nnz_c, nnz_f = results[-1]["nnz"], results[-1]["nnz_full"]
     sym_ms = np.mean([B.spsyrk_plan_timings(r["plan"])[0] for r in results], axis=0)
     num_ms = np.mean([B.spsyrk_plan_timings(r["plan"])[1] for r in results], axis=0)
-    value = whole_job_rate(work_total, world, ms_per_step)
+    if shard:
+        work_total = int(sum_over_ranks(work_total, "cuda"))
+        nnz_c = int(sum_over_ranks(nnz_c, "cuda"))
+        value = whole_job_rate(work_total, 1, ms_per_step)
+    else:
+        value = whole_job_rate(work_total, world, ms_per_step)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dname,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if shard else "weak", "vs_baseline": None, "dtype": dname,
             "data": "synthetic",
             "config": {"workload": a.name, "m": a.m, "n": a.n, "nnz_a": a.nnz, "multiply_adds": work_total, "nnz_c_l": nnz_c,
                        "nnz_full": nnz_f, "step": "plan+symbolic+numeric" + ("+mirror" if do_mirror else "") + ("+jaccard" if is_int else ""),
-                       "l2_policy": "inputs_larger_than_l2", "parallelism": f"replicas x{world}"},
-            "nnz_per_s": whole_job_rate(nnz_c, world, ms_per_step), "phases_ms": phases,
+                       "l2_policy": "inputs_larger_than_l2", "parallelism": f"rows x{world}" if shard else f"replicas x{world}"},
+            "nnz_per_s": whole_job_rate(nnz_c, 1 if shard else world, ms_per_step), "phases_ms": phases,
             "numeric_class_ms": [float(x) for x in num_ms], "symbolic_class_ms": [float(x) for x in sym_ms],
             "class_rows": class_rows, "gpu_launches": int(launches), "clocks": clocks}
 
+    if shard:
+        line["allgather_ms"] = allgather_ms
+        if rank == 0:
+            print(json.dumps(line))
+        dist.destroy_process_group()
+        return
     if rank == 0 and not args.skip_extras:
         # ---- roofline of the dominant kernel (the numeric launch of the heaviest row class)
         peak, peak_kind = measured_peaks()
@@ -501,6 +550,8 @@ def main():
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--rmat-noperm", action="store_true", help="with --rmat-scale: skip the random relabelling (load-balance study)")
+    ap.add_argument("--shard-rows", action="store_true",
+                    help="N > 1 only: one product, output rows split over the ranks by equal work (default: N replicas)")
     ap.add_argument("--skip-extras", action="store_true", help="timed steps only (for profiler runs)")
     ap.add_argument("--zipf-rows", type=int, default=0,
                     help="profiling aid: replace the workload by the binary Zipf recipe with this many rows")
