@@ -323,8 +323,11 @@ const char *spsyrk_status_string(spsyrk_status_t s);
  *      device state in *session.
  *   2. with h_c_colidx / h_c_vals of *nnz_out entries: runs numeric, copies the result back and
  *      frees the session.
- * Device memory for this entry point is allocated and freed by the library (cudaMalloc).
- * Host buffers should be pinned for full copy speed.  Synchronous.
+ * Device memory for this entry point is allocated by the library (cudaMalloc) and kept in two
+ * grow-only blocks per device between calls, because allocating and freeing several GB per call
+ * costs more than the computation; spsyrk_host_release_cache frees the blocks of the current
+ * device that no live session uses.  A call made while another thread's session holds the blocks
+ * allocates and frees its own.  Host buffers should be pinned for full copy speed.  Synchronous.
  */
 typedef struct spsyrk_session_s *spsyrk_session_t;
 spsyrk_status_t spsyrk_host_tril(spsyrk_session_t *session, int64_t m, int64_t n, int64_t nnz,
@@ -332,6 +335,7 @@ spsyrk_status_t spsyrk_host_tril(spsyrk_session_t *session, int64_t m, int64_t n
                                  spsyrk_dtype_t dtype, spsyrk_mode_t mode,
                                  int64_t *h_c_rowptr, int64_t *nnz_out,
                                  int32_t *h_c_colidx, void *h_c_vals);
+spsyrk_status_t spsyrk_host_release_cache(void);
 
 #ifdef __cplusplus
 }

@@ -45,6 +45,7 @@ _lib.spsyrk_column_panel.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _i64, _i64
 _lib.spsyrk_accumulate.argtypes = [_i64, _int, _i64, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_permute.argtypes = [_i64, _i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _szp, _vp]
 _lib.spsyrk_plan_partition.argtypes = [_vp, _i64, _i64p, _vp]
+_lib.spsyrk_host_release_cache.argtypes = []
 _lib.spsyrk_mirror_rowptr_noalloc.argtypes = [_i64, _vp, _vp, _vp, _i64p, _vp]
 _lib.spsyrk_mirror_rowptr_noalloc.restype = _int
 _lib.spsyrk_symv.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -65,7 +66,7 @@ for _name in ("spsyrk_plan_enable_timing", "spsyrk_plan_timings"):
     getattr(_lib, _name).restype = _int
 for _name in ("spsyrk_plan", "spsyrk_plan_set_rows", "spsyrk_symbolic", "spsyrk_numeric", "spsyrk_mirror",
               "spsyrk_jaccard", "spsyrk_plan_stats", "spsyrk_plan_buffers", "spsyrk_host_tril", "spsyrk_column_panel",
-              "spsyrk_accumulate", "spsyrk_permute", "spsyrk_plan_partition"):
+              "spsyrk_accumulate", "spsyrk_permute", "spsyrk_plan_partition", "spsyrk_host_release_cache"):
     getattr(_lib, _name).restype = _int
 
 
@@ -396,6 +397,11 @@ def spsyrk_host_tril(m, n, rowptr, colidx, vals, mode=TRIL, pinned=True, out=Non
     _check(_lib.spsyrk_host_tril(ctypes.byref(sess), m, n, nnz, None, None, None, code, mode, None, None,
                                  _p(c_colidx), _p(c_vals)), "spsyrk_host_tril(numeric)")
     return c_rowptr, c_colidx[:nnz_c.value], c_vals[:nnz_c.value]
+
+
+def spsyrk_host_release_cache():
+    """Free the device blocks spsyrk_host_tril keeps between calls on the current device."""
+    _check(_lib.spsyrk_host_release_cache(), "spsyrk_host_release_cache")
 
 
 # ------------------------------------------------------------------------------------------

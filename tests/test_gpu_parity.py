@@ -241,6 +241,21 @@ def test_host_entry_point(B):
     check_values(cv.numpy(), ref, a.vals.dtype)
 
 
+def test_host_entry_point_reuses_its_device_blocks(B):
+    """Calls of different sizes in a row (the cached blocks grow, then serve a smaller problem), a
+    release in between, and a mode change: results stay those of the oracle."""
+    for idx, mode in [(1, 0), (5, 0), (1, 1), (3, 0)]:
+        if idx == 3:
+            B.spsyrk_host_release_cache()
+        a = W.small(idx)
+        rp, ci, cv = B.spsyrk_host_tril(a.m, a.n, torch.from_numpy(a.rowptr), torch.from_numpy(a.colidx),
+                                        torch.from_numpy(a.vals), mode=mode)
+        ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, mode)
+        assert np.array_equal(rp.numpy(), ref.rowptr) and np.array_equal(ci.numpy(), ref.colidx)
+        check_values(cv.numpy(), ref, a.vals.dtype)
+    B.spsyrk_host_release_cache()
+
+
 # ------------------------------------------------------------------ further dtypes and error paths
 def test_int32_general_values_and_fp32_light_rows(B):
     rng = np.random.default_rng(11)
