@@ -144,11 +144,14 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
             if (tid == 0) loff[THREADS] = T;
             if (is_long) long_idx[atomicAdd(&s_nlong, 1u)] = tid;
             __syncthreads();
-            // short lists, flattened: every thread takes a contiguous run of items (so that moving
-            // from one list to the next is a step, not a search), UNR loads in flight at a time
+            // short lists, flattened: every warp takes a contiguous run of items and its lanes interleave
+            // inside it, so that a warp's loads are coalesced and UNR different lines are in flight; a lane
+            // steps from list to list as its items advance (no search per item)
             {
-                const uint32_t ipt = (T + THREADS - 1) / THREADS;
-                const uint32_t first = min((uint32_t)tid * ipt, T), last = min(first + ipt, T);
+                constexpr uint32_t NW = THREADS / 32;
+                const uint32_t per_warp = ((T + NW - 1) / NW + 31u) & ~31u;
+                const uint32_t wfirst = min((uint32_t)(tid >> 5) * per_warp, T), last = min(wfirst + per_warp, T);
+                const uint32_t first = wfirst + (tid & 31);
                 if (first < last) {
                     uint32_t lo_l = 0, hi_l = THREADS;  // last list whose offset is <= first
                     while (hi_l - lo_l > 1) {
@@ -157,12 +160,12 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     }
                     uint32_t cur = lo_l, cur_off = loff[cur], next_off = loff[cur + 1], cur_start = lstart[cur];
                     Acc cur_a = WHAT == CTA_ACCUM ? la[cur] : Acc(0);
-                    for (uint32_t item0 = first; item0 < last; item0 += UNR) {
+                    for (uint32_t item0 = first; item0 < last; item0 += UNR * 32) {
                         uint32_t q[UNR];
                         Acc av[UNR];
 #pragma unroll
                         for (int u = 0; u < UNR; ++u) {
-                            const uint32_t item = item0 + u;
+                            const uint32_t item = item0 + u * 32;
                             q[u] = 0xffffffffu;
                             av[u] = Acc(0);
                             if (item < last) {
