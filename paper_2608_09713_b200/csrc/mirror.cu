@@ -72,10 +72,16 @@ __global__ void __launch_bounds__(256) mirror_count_kernel(const int64_t* __rest
     const int gl = threadIdx.x & (G - 1);
     if (r >= m) return;
     const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
-    for (int64_t p = p0 + gl; p < p1; p += G) {
-        const int64_t j = l_colidx[p];
-        if (j > r || j < 0) atomicOr(err, ERRW_UPPER);
-        else if (j < r) atomicAdd(&ucnt[j], 1u);
+    constexpr int UNR = 4;
+    for (int64_t p = p0 + gl; p < p1; p += UNR * G) {
+        int64_t j[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) j[u] = p + u * G < p1 ? (int64_t)l_colidx[p + u * G] : r;  // r: neither counted nor an error
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            if (j[u] > r || j[u] < 0) atomicOr(err, ERRW_UPPER);
+            else if (j[u] < r) atomicAdd(&ucnt[j[u]], 1u);
+        }
     }
 }
 
@@ -97,12 +103,28 @@ __global__ void __launch_bounds__(256) mirror_expand_kernel(const int64_t* __res
     if (r >= m) return;
     const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
     const int64_t fb = f_rowptr[r];
-    for (int64_t p = p0 + gl; p < p1; p += G) {
-        const int32_t j = l_colidx[p];
-        f_colidx[fb + (p - p0)] = j;
-        f_vals[fb + (p - p0)] = l_vals[p];
-        key0[p] = j == r ? (uint32_t)m : (uint32_t)j;
-        row0[p] = (uint32_t)r;
+    constexpr int UNR = 4;  // loads of several steps are issued before the first store
+    for (int64_t p = p0 + gl; p < p1; p += UNR * G) {
+        int32_t j[UNR];
+        V v[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int64_t pp = p + u * G;
+            if (pp < p1) {
+                j[u] = l_colidx[pp];
+                v[u] = l_vals[pp];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int64_t pp = p + u * G;
+            if (pp < p1) {
+                f_colidx[fb + (pp - p0)] = j[u];
+                f_vals[fb + (pp - p0)] = v[u];
+                key0[pp] = j[u] == r ? (uint32_t)m : (uint32_t)j[u];
+                row0[pp] = (uint32_t)r;
+            }
+        }
     }
 }
 

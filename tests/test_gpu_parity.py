@@ -212,6 +212,40 @@ def test_mirror_rejects_upper_entries(B):
     assert e.value.status == 2
 
 
+@pytest.mark.parametrize("m,density,diag", [(7, 0.5, "some"), (200, 0.1, "some"), (200, 0.1, "none"), (3000, 0.004, "all"),
+                                            (70000, 0.0001, "some")])
+def test_mirror_general_lower_triangles(B, m, density, diag):
+    """Lower triangles that are not products: rows without a diagonal entry, empty rows, one pass
+    (m < 256) up to three radix passes (m > 65536)."""
+    rng = np.random.default_rng(m)
+    nnz_target = int(density * m * m / 2) + m
+    r = rng.integers(0, m, size=nnz_target)
+    c = (rng.random(nnz_target) * (r + 1)).astype(np.int64)     # c <= r
+    keep = c < r
+    r, c = r[keep], c[keep]
+    if diag != "none":
+        d = np.arange(m) if diag == "all" else rng.choice(m, size=m // 2, replace=False)
+        r, c = np.concatenate([r, d]), np.concatenate([c, d])
+    key = np.unique(r * m + c)
+    r, c = key // m, key % m
+    rp = np.zeros(m + 1, dtype=np.int64)
+    np.cumsum(np.bincount(r, minlength=m), out=rp[1:])
+    vals = rng.standard_normal(c.size)
+    got = B.spsyrk_mirror(m, torch.from_numpy(rp).cuda(), torch.from_numpy(c.astype(np.int32)).cuda(), torch.from_numpy(vals).cuda())
+    exp = oracle.mirror(m, rp, c.astype(np.int32), vals)
+    for g, e in zip(got, exp):
+        assert np.array_equal(g.cpu().numpy(), e)
+
+
+def test_mirror_of_nothing(B):
+    z = (torch.zeros(1, dtype=torch.int64, device="cuda"), torch.zeros(0, dtype=torch.int32, device="cuda"),
+         torch.zeros(0, dtype=torch.float64, device="cuda"))
+    assert B.spsyrk_mirror(0, *z)[0].cpu().tolist() == [0]
+    z5 = (torch.zeros(6, dtype=torch.int64, device="cuda"), z[1], z[2])
+    f = B.spsyrk_mirror(5, *z5)
+    assert f[0].cpu().tolist() == [0] * 6 and f[1].numel() == 0
+
+
 # ---------------------------------------------------------------------------------- jaccard
 def test_jaccard(B):
     a = W.small(2)
