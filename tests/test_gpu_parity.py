@@ -263,6 +263,18 @@ def test_jaccard(B):
     trp, tci, tcv, _ = B.tril_syrk(a.m, a.n, *dev(a), row_begin=r0, row_end=r1, plan=plan)
     tj = B.spsyrk_jaccard(a.m, r0, r1 - r0, rowptr_a, trp, tci, tcv).cpu().numpy()
     assert np.array_equal(tj, exp[ref.rowptr[r0]:ref.rowptr[r1]])
+    # arrays that do not start on 16 bytes take the scalar path; short rows straddle the 4-entry steps
+    def shifted(t):
+        buf = torch.empty(t.numel() + 1, dtype=t.dtype, device=t.device)
+        buf[1:].copy_(t)
+        return buf[1:]
+    out = shifted(torch.zeros(ci.numel(), dtype=torch.float32, device="cuda"))
+    uj = B.spsyrk_jaccard(a.m, 0, a.m, rowptr_a, rp, shifted(ci), shifted(cv), out=out).cpu().numpy()
+    assert np.array_equal(uj, exp)
+    b = W.small(4)                                            # binary values, about 50 entries per output row
+    (rp4, ci4, cv4), ref4, _ = run_and_compare(B, W.CSR(b.m, b.n, b.rowptr, b.colidx, np.ones(b.nnz, dtype=np.int32)), 0)
+    j4 = B.spsyrk_jaccard(b.m, 0, b.m, torch.from_numpy(b.rowptr).cuda(), rp4, ci4, cv4).cpu().numpy()
+    assert np.array_equal(j4, oracle.jaccard(0, b.m, b.rowptr, ref4.rowptr, ref4.colidx, oracle.to_int32(ref4.vals)))
 
 
 # --------------------------------------------------------------------- host-buffer entry point
