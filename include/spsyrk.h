@@ -140,11 +140,17 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t *d_c_rowptr,
  * every later row r that stores column i, ascending in r; values are bit copies, so F is
  * exactly symmetric and tril(F) == C_L.
  *
+ * C_L must have its rows ascending in column, as spsyrk_numeric writes them.
+ *
  * Three-step use:
  *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for (m, nnz_l, dtype).
- *   2. d_f_colidx == NULL: writes d_f_rowptr[m + 1] and *nnz_full_out (synchronises).
- *   3. all pointers set: fills d_f_colidx / d_f_vals using the d_f_rowptr of step 2.  Asynchronous.
- * nnz_l = d_l_rowptr[m].  d_l_vals must be 16-byte aligned.  Errors: INVALID_ARG, WORKSPACE, BAD_CSR (an entry above the diagonal), CUDA.
+ *   2. d_f_colidx == NULL: looks at the first and last entry of every row (with ascending rows that
+ *      finds any entry above the diagonal and every stored diagonal) and returns
+ *      *nnz_full_out = 2 nnz_l - #diagonal entries (synchronises).  d_f_rowptr is not written yet.
+ *   3. all pointers set: writes d_f_rowptr[m + 1] and fills d_f_colidx / d_f_vals (nnz_full entries).
+ *      Asynchronous.  An entry above the diagonal that step 2 could not see (a row that is not
+ *      ascending) is left out of the reflection; it never indexes outside the arrays.
+ * nnz_l = d_l_rowptr[m].  Errors: INVALID_ARG, WORKSPACE, BAD_CSR (an entry above the diagonal), CUDA.
  */
 spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
                               const int64_t *d_l_rowptr, const int32_t *d_l_colidx, const void *d_l_vals,

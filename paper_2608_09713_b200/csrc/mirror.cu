@@ -3,14 +3,18 @@
 // Row j of F = row j of C_L (columns <= j) followed by the reflected entries (r, c_rj) of the
 // later rows r > j that store column j, ascending in r.  That second part is a transpose of the
 // strictly lower triangle, done as a stable radix sort of the entries by column id:
-//   count   : per column j the number of strictly lower entries (atomics), add the row's own
-//             length, scan -> f_rowptr.
-//   expand  : copy the lower parts into F; write an explicit (key, row) pair per entry, the key
-//             being the column id, or m for a diagonal entry so that diagonals sort past the end.
+//   sizes   : rows are ascending, so a row stores its diagonal iff its last entry is the diagonal and
+//             holds an entry above the diagonal iff its last entry is one:
+//             nnz(F) = 2 nnz(C_L) - #diagonals.
+//   expand  : an explicit (key, row) pair per entry, the key being the column id, or m for a
+//             diagonal entry (and for an entry that should not be there) so that it sorts past the end.
 //   sort    : stable LSD radix passes over (key, row, value); entries enter in ascending row order,
 //             so every column's segment comes out ascending in r.  The last pass writes straight
 //             into F: the s-th strictly lower entry in sorted order, of column j, lands at
-//             s + l_rowptr[j + 1].
+//             s + l_rowptr[j + 1].  It also records where each column's segment starts and ends
+//             (equal keys are adjacent in the last pass: one atomic at each end of a run), which is
+//             the number of reflected entries of row j.
+//   rows    : row lengths of F, scan -> f_rowptr, then the lower parts are copied into place.
 #include <algorithm>
 #include <mutex>
 
@@ -25,8 +29,10 @@ constexpr size_t ALIGN = 256;
 constexpr int MIRROR_RADIX_BITS = 8;
 
 struct MirrorWs {
-    uint32_t* ucnt;    // m: strictly-lower entries per column
+    uint32_t* ucnt;    // m: strictly-lower entries per column (allocation-free size step only)
     uint32_t* rowtot;  // m
+    unsigned long long* seg_start;  // m: first sorted position of column j's strictly lower entries
+    unsigned long long* seg_end;    // m: one past the last
     int64_t* partials;
     uint32_t* err;
     // radix sort buffers (nnz_l entries each); buffer B's key and row arrays double as the expanded input
@@ -51,8 +57,10 @@ size_t carve(MirrorWs* w, void* ws, int64_t m, int64_t nnz_l, size_t sv) {
     MirrorWs t;
     t.ucnt = (uint32_t*)take(items * 4);
     t.rowtot = (uint32_t*)take(items * 4);
+    t.seg_start = (unsigned long long*)take(items * 8);
+    t.seg_end = (unsigned long long*)take(items * 8);
     t.partials = (int64_t*)take(scan_partials_count(std::max<int64_t>(items + 1, hist_n)) * 8);
-    t.err = (uint32_t*)take(4);
+    t.err = (uint32_t*)take(8);  // [0] error word, [1] number of diagonal entries
     t.key_a = (uint32_t*)take(ne * 4);
     t.row_a = (uint32_t*)take(ne * 4);
     t.key_b = (uint32_t*)take(ne * 4);
@@ -91,19 +99,60 @@ __global__ void mirror_rowtot_kernel(const int64_t* __restrict__ l_rowptr, const
     if (r < m) rowtot[r] = (uint32_t)(l_rowptr[r + 1] - l_rowptr[r]) + ucnt[r];
 }
 
-// G lanes per row: copy the row into F and write the explicit (key, row) pair of every entry.
-template <typename V, int G>
+// one thread per row: the last entry tells whether the row stores its diagonal and whether it reaches above it
+// (rows are ascending); err[1] counts the diagonals
+__global__ void mirror_last_entry_kernel(const int64_t* __restrict__ l_rowptr, const int32_t* __restrict__ l_colidx, int64_t m,
+                                         uint32_t* err) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= m) return;
+    const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
+    if (p1 < p0) { atomicOr(err, ERRW_BAD_ROWPTR); return; }
+    if (p1 == p0) return;
+    const int64_t last = l_colidx[p1 - 1], first = l_colidx[p0];
+    if (last > r || first < 0) atomicOr(err, ERRW_UPPER);
+    else if (last == r) atomicAdd(err + 1, 1u);
+}
+
+// G lanes per row: the explicit (key, row) pair of every entry
+template <int G>
 __global__ void __launch_bounds__(256) mirror_expand_kernel(const int64_t* __restrict__ l_rowptr, const int32_t* __restrict__ l_colidx,
-                                                            const V* __restrict__ l_vals, int64_t m,
-                                                            const int64_t* __restrict__ f_rowptr, int32_t* __restrict__ f_colidx,
-                                                            V* __restrict__ f_vals, uint32_t* __restrict__ key0,
-                                                            uint32_t* __restrict__ row0) {
+                                                            int64_t m, uint32_t* __restrict__ key0, uint32_t* __restrict__ row0,
+                                                            uint32_t* err) {
     const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
     const int gl = threadIdx.x & (G - 1);
     if (r >= m) return;
     const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
-    const int64_t fb = f_rowptr[r];
     constexpr int UNR = 4;  // loads of several steps are issued before the first store
+    for (int64_t p = p0 + gl; p < p1; p += UNR * G) {
+        int64_t j[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) j[u] = p + u * G < p1 ? (int64_t)l_colidx[p + u * G] : r;
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int64_t pp = p + u * G;
+            if (pp < p1) {
+                // an entry outside the lower triangle (rows that are not ascending can hide one from the size
+                // step) is keyed like a diagonal: it takes no part in the reflection
+                if (j[u] > r || j[u] < 0) atomicOr(err, ERRW_UPPER);
+                key0[pp] = (j[u] >= r || j[u] < 0) ? (uint32_t)m : (uint32_t)j[u];
+                row0[pp] = (uint32_t)r;
+            }
+        }
+    }
+}
+
+// G lanes per row: the lower part of row r of F is row r of C_L
+template <typename V, int G>
+__global__ void __launch_bounds__(256) mirror_copy_lower_kernel(const int64_t* __restrict__ l_rowptr, const int32_t* __restrict__ l_colidx,
+                                                                const V* __restrict__ l_vals, int64_t m,
+                                                                const int64_t* __restrict__ f_rowptr, int32_t* __restrict__ f_colidx,
+                                                                V* __restrict__ f_vals) {
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    const int gl = threadIdx.x & (G - 1);
+    if (r >= m) return;
+    const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
+    const int64_t fb = f_rowptr[r] - p0;
+    constexpr int UNR = 4;
     for (int64_t p = p0 + gl; p < p1; p += UNR * G) {
         int32_t j[UNR];
         V v[UNR];
@@ -119,26 +168,39 @@ __global__ void __launch_bounds__(256) mirror_expand_kernel(const int64_t* __res
         for (int u = 0; u < UNR; ++u) {
             const int64_t pp = p + u * G;
             if (pp < p1) {
-                f_colidx[fb + (pp - p0)] = j[u];
-                f_vals[fb + (pp - p0)] = v[u];
-                key0[pp] = j[u] == r ? (uint32_t)m : (uint32_t)j[u];
-                row0[pp] = (uint32_t)r;
+                f_colidx[fb + pp] = j[u];
+                f_vals[fb + pp] = v[u];
             }
         }
     }
 }
 
+// row lengths of F: the row's own entries plus the length of its column's sorted segment
+__global__ void mirror_rowlen_kernel(const int64_t* __restrict__ l_rowptr, const unsigned long long* __restrict__ seg_start,
+                                     const unsigned long long* __restrict__ seg_end, int64_t m, uint32_t* __restrict__ rowtot) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= m) return;
+    const unsigned long long s = seg_start[r], e = seg_end[r];
+    rowtot[r] = (uint32_t)(l_rowptr[r + 1] - l_rowptr[r]) + (e > s ? (uint32_t)(e - s) : 0u);
+}
+
 template <typename V>
 struct EmitMirrorFinal {
+    static constexpr bool NEIGHBOURS = true;
     const int64_t* l_rowptr;
     int32_t* f_colidx;
     V* f_vals;
+    unsigned long long* seg_start;
+    unsigned long long* seg_end;
     uint32_t m;
-    __device__ __forceinline__ void operator()(int64_t dest, uint32_t key, uint32_t row, V val) const {
+    __device__ __forceinline__ void operator()(int64_t dest, uint32_t key, uint32_t row, V val, uint32_t prev, uint32_t next) const {
         if (key < m) {  // diagonal entries were keyed m and are dropped here
             const int64_t pos = dest + l_rowptr[key + 1];
             f_colidx[pos] = (int32_t)row;
             f_vals[pos] = val;
+            // ends of a run of one key inside the tile; a segment that spans tiles settles through min / max
+            if (prev != key) atomicMin(&seg_start[key], (unsigned long long)dest);
+            if (next != key) atomicMax(&seg_end[key], (unsigned long long)dest + 1ull);
         }
     }
 };
@@ -150,42 +212,65 @@ int group_width(int64_t nnz, int64_t m) {
 
 template <typename V>
 spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const int64_t* l_rowptr, const int32_t* l_colidx,
-                            const void* l_vals, const int64_t* f_rowptr, int32_t* f_colidx, void* f_vals, cudaStream_t st) {
+                            const void* l_vals, int64_t* f_rowptr, int32_t* f_colidx, void* f_vals, cudaStream_t st) {
     constexpr int BITS = MIRROR_RADIX_BITS;
     const V* lv = static_cast<const V*>(l_vals);
     V* fv = static_cast<V*>(f_vals);
-#define EXPAND(G)                                                                                                   \
-    mirror_expand_kernel<V, G><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(l_rowptr, l_colidx, lv, m, f_rowptr, \
-                                                                                f_colidx, fv, w.key_b, w.row_b)
-    switch (group_width(nnz_l, m)) {
-        case 4: EXPAND(4); break;
-        case 8: EXPAND(8); break;
-        case 16: EXPAND(16); break;
-        default: EXPAND(32); break;
+    const int g = group_width(nnz_l, m);
+    if (m > 0) {
+        SPSYRK_CUDA_TRY(cudaMemsetAsync(w.seg_start, 0xff, (size_t)m * 8, st));
+        SPSYRK_CUDA_TRY(cudaMemsetAsync(w.seg_end, 0, (size_t)m * 8, st));
     }
-#undef EXPAND
-    note_launches(1);
-    if (nnz_l == 0) return SPSYRK_OK;
-    const int npass = (bits_for((uint64_t)m) + BITS - 1) / BITS;  // keys run from 0 to m
-    const uint32_t* src_key = w.key_b;
-    const uint32_t* src_row = w.row_b;
-    const V* src_val = lv;
-    for (int p = 0; p < npass; ++p) {
-        const bool to_a = (p % 2) == 0;
-        uint32_t* dst_key = to_a ? w.key_a : w.key_b;
-        uint32_t* dst_row = to_a ? w.row_a : w.row_b;
-        V* dst_val = static_cast<V*>(to_a ? w.val_a : w.val_b);
-        if (p == npass - 1) {
-            EmitMirrorFinal<V> emit{l_rowptr, f_colidx, fv, (uint32_t)m};
-            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
-        } else {
-            EmitArrays<V> emit{dst_key, dst_row, dst_val};
-            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+    if (m > 0 && nnz_l > 0) {
+#define EXPAND(G) mirror_expand_kernel<G><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(l_rowptr, l_colidx, m, w.key_b, w.row_b, w.err)
+        switch (g) {
+            case 4: EXPAND(4); break;
+            case 8: EXPAND(8); break;
+            case 16: EXPAND(16); break;
+            default: EXPAND(32); break;
         }
-        src_key = dst_key;
-        src_row = dst_row;
-        src_val = dst_val;
+#undef EXPAND
+        note_launches(1);
+        const int npass = (bits_for((uint64_t)m) + BITS - 1) / BITS;  // keys run from 0 to m
+        const uint32_t* src_key = w.key_b;
+        const uint32_t* src_row = w.row_b;
+        const V* src_val = lv;
+        for (int p = 0; p < npass; ++p) {
+            const bool to_a = (p % 2) == 0;
+            uint32_t* dst_key = to_a ? w.key_a : w.key_b;
+            uint32_t* dst_row = to_a ? w.row_a : w.row_b;
+            V* dst_val = static_cast<V*>(to_a ? w.val_a : w.val_b);
+            if (p == npass - 1) {
+                EmitMirrorFinal<V> emit{l_rowptr, f_colidx, fv, w.seg_start, w.seg_end, (uint32_t)m};
+                SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+            } else {
+                EmitArrays<V> emit{dst_key, dst_row, dst_val};
+                SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+            }
+            src_key = dst_key;
+            src_row = dst_row;
+            src_val = dst_val;
+        }
     }
+    // row pointers of F, then the lower parts
+    if (m > 0) {
+        mirror_rowlen_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(l_rowptr, w.seg_start, w.seg_end, m, w.rowtot);
+        note_launches(1);
+    }
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(w.rowtot, m, f_rowptr, w.partials, st));
+    if (m > 0 && nnz_l > 0) {
+#define COPY(G) \
+    mirror_copy_lower_kernel<V, G><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(l_rowptr, l_colidx, lv, m, f_rowptr, f_colidx, fv)
+        switch (g) {
+            case 4: COPY(4); break;
+            case 8: COPY(8); break;
+            case 16: COPY(16); break;
+            default: COPY(32); break;
+        }
+#undef COPY
+        note_launches(1);
+    }
+    SPSYRK_CUDA_TRY(cudaGetLastError());
     return SPSYRK_OK;
 }
 
@@ -211,36 +296,22 @@ extern "C" spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_
     MirrorWs w;
     carve(&w, d_workspace, m, nnz_l, sv);
 
-    if (!d_f_colidx) {  // step 2: sizes
+    if (!d_f_colidx) {  // step 2: checks and nnz(F)
         if (!nnz_full_out) return SPSYRK_ERR_INVALID_ARG;
-        SPSYRK_CUDA_TRY(cudaMemsetAsync(w.err, 0, 4, st));
+        SPSYRK_CUDA_TRY(cudaMemsetAsync(w.err, 0, 8, st));
         if (m > 0) {
-            SPSYRK_CUDA_TRY(cudaMemsetAsync(w.ucnt, 0, (size_t)m * 4, st));
-#define COUNT(G) mirror_count_kernel<G><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(d_l_rowptr, d_l_colidx, m, w.ucnt, w.err)
-            switch (group_width(nnz_l, m)) {
-                case 4: COUNT(4); break;
-                case 8: COUNT(8); break;
-                case 16: COUNT(16); break;
-                default: COUNT(32); break;
-            }
-#undef COUNT
-            mirror_rowtot_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(d_l_rowptr, w.ucnt, m, w.rowtot);
-            note_launches(2);  // count + row totals
+            mirror_last_entry_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(d_l_rowptr, d_l_colidx, m, w.err);
+            note_launches(1);
         }
-        SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(w.rowtot, m, d_f_rowptr, w.partials, st));
-        int64_t nnz = 0;
-        uint32_t e = 0;
-        SPSYRK_CUDA_TRY(cudaMemcpyAsync(&nnz, d_f_rowptr + m, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
-        SPSYRK_CUDA_TRY(cudaMemcpyAsync(&e, w.err, 4, cudaMemcpyDeviceToHost, st));
+        uint32_t e[2] = {0, 0};
+        SPSYRK_CUDA_TRY(cudaMemcpyAsync(e, w.err, 8, cudaMemcpyDeviceToHost, st));
         SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
-        if (e & ERRW_UPPER) return SPSYRK_ERR_BAD_CSR;
-        *nnz_full_out = nnz;
+        if (e[0]) return SPSYRK_ERR_BAD_CSR;
+        *nnz_full_out = 2 * nnz_l - (int64_t)e[1];
         return SPSYRK_OK;
     }
     // step 3: fill
     if (!d_f_vals || (nnz_l > 0 && !d_l_vals)) return SPSYRK_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(d_l_vals) % 16) return SPSYRK_ERR_INVALID_ARG;  // tiles of it are copied 16 bytes at a time
-    if (m == 0) return SPSYRK_OK;
     switch (dtype) {
         case SPSYRK_F64: return mirror_fill<uint64_t>(w, m, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_f_rowptr, d_f_colidx, d_f_vals, st);
         default: return mirror_fill<uint32_t>(w, m, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_f_rowptr, d_f_colidx, d_f_vals, st);

@@ -11,6 +11,8 @@
 // digit-major tile in shared memory and the tile is written out in runs.  There is no waiting
 // between CTAs.
 #pragma once
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace spsyrk {
@@ -51,6 +53,14 @@ __global__ void __launch_bounds__(RX_THREADS) radix_hist_kernel(const uint32_t* 
         hist[(int64_t)d * ntiles + blockIdx.x] = t;
     }
 }
+
+// A functor that declares `static constexpr bool NEIGHBOURS = true` is also handed the keys next to the
+// element in the tile's sorted order.
+constexpr uint32_t NO_KEY = 0xffffffffu;
+template <typename E, typename = void>
+struct emit_wants_neighbours : std::false_type {};
+template <typename E>
+struct emit_wants_neighbours<E, std::void_t<decltype(E::NEIGHBOURS)>> : std::bool_constant<E::NEIGHBOURS> {};
 
 template <int BITS, typename PB>
 struct RadixSmem {
@@ -180,7 +190,14 @@ __global__ void __launch_bounds__(RX_THREADS, 2) radix_scatter_kernel(const uint
     __syncthreads();
     for (int q = tid; q < tile_n; q += RX_THREADS) {
         const uint32_t key = s_key[q];
-        emit(goff[(key >> shift) & (NB - 1)] + q, key, s_pa[q], s_pb[q]);
+        const int64_t dest = goff[(key >> shift) & (NB - 1)] + q;
+        if constexpr (emit_wants_neighbours<Emit>::value) {
+            // the keys of the slots before and after (NO_KEY at the ends of the tile): in the last pass of a
+            // sort equal keys are adjacent, so a functor can tell where a run of one key starts and ends
+            emit(dest, key, s_pa[q], s_pb[q], q > 0 ? s_key[q - 1] : NO_KEY, q + 1 < tile_n ? s_key[q + 1] : NO_KEY);
+        } else {
+            emit(dest, key, s_pa[q], s_pb[q]);
+        }
     }
 }
 
