@@ -147,3 +147,62 @@ def test_row_tiles_at_scale(B):
     assert torch.equal(torch.cat(counts), rp[1:] - rp[:-1])
     assert torch.equal(torch.cat(cols), ci)
     assert torch.equal(torch.cat(vals), cv)
+
+
+def test_panels_accumulate_to_the_whole_at_scale(B):
+    """The accumulating form on the large Erdos-Renyi configuration: two column panels, their products
+    summed; the structure must be that of the unsplit product bit for bit and the values agree to
+    rounding (both sides are sums of the same partial products, grouped differently)."""
+    a = W.config(5)
+    d = (torch.from_numpy(a.rowptr).cuda(), torch.from_numpy(a.colidx).cuda(), torch.from_numpy(a.vals).cuda())
+    rp, ci, cv, _ = B.tril_syrk(a.m, a.n, *d)
+    prods = []
+    for k0, k1 in ((0, a.n // 2), (a.n // 2, a.n)):
+        p = B.spsyrk_column_panel(a.m, *d, k0, k1)
+        prods.append(B.tril_syrk(a.m, a.n, *p)[:3])
+        del p
+    assert int(prods[0][1].numel()) + int(prods[1][1].numel()) >= int(ci.numel())
+    zr, zc, zv = B.spsyrk_accumulate(a.m, *prods[0], *prods[1])
+    del prods
+    torch.cuda.synchronize()
+    assert torch.equal(zr, rp) and torch.equal(zc, ci)
+    # |difference| <= 1e-12 * (sum of |partial products|) <= 1e-12 * 16 since values lie in [-1, 1) and rows hold 16 entries
+    assert float((zv - cv).abs().max()) <= 16e-12
+
+
+def test_permutation_at_scale(B):
+    """The symmetric permutation on the R-MAT configuration: sampled rows of the permuted matrix against
+    the definition, and the product of the permuted matrix has the nnz and the diagonal of the original."""
+    a = W.config(3)
+    rng = np.random.default_rng(77)
+    perm = rng.permutation(a.m).astype(np.int32)
+    d = (torch.from_numpy(a.rowptr).cuda(), torch.from_numpy(a.colidx).cuda(), torch.from_numpy(a.vals).cuda())
+    pt = torch.from_numpy(perm).cuda()
+    br, bc, bv = B.spsyrk_permute(a.m, a.n, *d, pt, pt)
+    brh = br.cpu().numpy()
+    assert np.array_equal(np.diff(brh)[perm], np.diff(a.rowptr))          # row i went to row perm[i] with its length
+    deg = np.diff(a.rowptr)
+    for i in sample_rows(a.m, deg, 40, 5):
+        src_c, src_v = a.colidx[a.rowptr[i]:a.rowptr[i + 1]], a.vals[a.rowptr[i]:a.rowptr[i + 1]]
+        order = np.argsort(perm[src_c], kind="stable")
+        lo, hi = int(brh[perm[i]]), int(brh[perm[i] + 1])
+        assert np.array_equal(bc[lo:hi].cpu().numpy(), perm[src_c][order])
+        assert np.array_equal(bv[lo:hi].cpu().numpy(), src_v[order])
+    rp, ci, cv, _ = B.tril_syrk(a.m, a.n, *d)
+    prp, pci, pcv, plan = B.tril_syrk(a.m, a.n, br, bc, bv)
+    # (P A P^T)(P A P^T)^T = P (A A^T) P^T: the lower triangles differ, the full products are permutations of each
+    # other, so nnz(tril) (every off-diagonal pair is stored once either way) and the diagonal values carry over
+    assert int(pci.numel()) == int(ci.numel())
+    diag = cv[(rp[1:] - 1).clamp(min=0)][torch.from_numpy(deg > 0).cuda()]
+    pdeg = torch.from_numpy(np.diff(brh) > 0).cuda()
+    pdiag = pcv[(prp[1:] - 1).clamp(min=0)][pdeg]
+    inv = torch.from_numpy(np.argsort(perm)).cuda()        # row r of the permuted matrix is row inv[r] of the original
+    full_diag = torch.zeros(a.m, dtype=cv.dtype, device="cuda")
+    full_diag[torch.from_numpy(deg > 0).cuda()] = diag
+    full_pdiag = torch.zeros(a.m, dtype=cv.dtype, device="cuda")
+    full_pdiag[pdeg] = pdiag
+    # a column permutation reorders the additions of each squared norm: equal to rounding
+    assert float((full_pdiag - full_diag[inv]).abs().max()) <= 1e-5 * float(full_diag.abs().max())
+    # equal-work row ranges of the plan tile the rows
+    b = B.spsyrk_plan_partition(plan, 8)
+    assert b[0] == 0 and b[-1] == a.m and all(x <= y for x, y in zip(b, b[1:]))
