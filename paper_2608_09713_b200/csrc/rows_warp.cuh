@@ -19,7 +19,7 @@ __host__ __device__ constexpr int symbolic_warps(int n) { return n >= 512 ? 4 : 
 // warps per CTA of the numeric warp-class kernel: keeps static shared memory under 48 KB
 __host__ __device__ constexpr int numeric_warps(int n) { return n >= 512 ? 2 : n >= 256 ? 4 : 8; }
 // register budget: at least this many CTAs of the numeric kernel must fit on an SM
-__host__ __device__ constexpr int numeric_min_ctas(int n) { return n == 256 ? 6 : 1; }
+__host__ __device__ constexpr int numeric_min_ctas(int n) { return n == 256 ? 6 : n == 128 ? 4 : n == 64 ? 5 : 1; }
 
 // lane holding the s-th (0-based) set bit of mask
 __device__ __forceinline__ uint32_t nth_set_lane(unsigned mask, uint32_t s) {
