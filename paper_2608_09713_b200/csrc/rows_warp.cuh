@@ -149,9 +149,7 @@ __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N)) nu
                 key[r] = ((Key)j << IDXB) | (Key)t;
             }
         }
-#ifndef EXPERIMENT_NOSORT
         group_bitonic_sort<Key, R, 32>(key);
-#endif
         __syncwarp();
 
         // same[r]: element r continues the run of equal j of element r-1 (same[0]: of the previous
