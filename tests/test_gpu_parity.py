@@ -582,3 +582,47 @@ def test_plan_partition(B, idx):
     assert np.array_equal(np.concatenate(pieces), whole.colidx)
     with pytest.raises(B.SpsyrkError):
         B.spsyrk_plan_partition(plan, 0)
+
+
+# ------------------------------------------------------------------ rows exactly at the class boundaries
+def test_rows_at_every_class_boundary(B):
+    """One column shared by all rows: row i has exactly i + 1 partial products and i + 1 output entries,
+    so consecutive rows walk through every class boundary (32|33, 64|65, ..., 512|513, 16384|16385).
+    Structure by closed form for every row, values (single products, exact) for every entry, and rows
+    around the boundaries against the oracle."""
+    m = 16500
+    rng = np.random.default_rng(3)
+    vals = rng.standard_normal(m)
+    a = W.CSR(m, 1, np.arange(m + 1, dtype=np.int64), np.zeros(m, dtype=np.int32), vals)
+    rp, ci, cv, plan = B.tril_syrk(a.m, a.n, *dev(a))
+    i = np.arange(m + 1, dtype=np.int64)
+    assert np.array_equal(rp.cpu().numpy(), i * (i + 1) // 2)
+    work, classes = B.spsyrk_plan_stats(plan)
+    assert work == m * (m + 1) // 2
+    assert classes == [0, 32, 32, 64, 128, 256, 16384 - 512, m - 16384]
+    rows = torch.repeat_interleave(torch.arange(m, device="cuda"), torch.arange(1, m + 1, device="cuda"))
+    cols = torch.arange(ci.numel(), device="cuda") - rp[:-1][rows]
+    assert torch.equal(ci.long(), cols)
+    v = torch.from_numpy(vals).cuda()
+    assert torch.equal(cv, v[rows] * v[cols])                 # one product per entry: no rounding to differ in
+    for r in (0, 31, 32, 63, 64, 127, 128, 255, 256, 511, 512, 16383, 16384, m - 1):
+        ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, r, r + 1)
+        lo, hi = int(rp[r]), int(rp[r + 1])
+        assert np.array_equal(ci[lo:hi].cpu().numpy(), ref.colidx)
+        assert np.array_equal(cv[lo:hi].cpu().numpy(), ref.vals)
+
+
+def test_rows_with_33_nonzeros_leave_the_warp_classes(B):
+    """At most 32 nonzeros fit the one-warp kernels: a row with 33 goes to the CTA kernels whatever its work."""
+    m, n = 40, 33
+    rng = np.random.default_rng(4)
+    dense = rng.standard_normal((m, n))
+    dense[::2, 32] = 0.0                                     # every other row has 32 nonzeros, the rest 33
+    rr, cc = np.nonzero(dense)
+    rowptr = np.zeros(m + 1, dtype=np.int64)
+    np.cumsum(np.bincount(rr, minlength=m), out=rowptr[1:])
+    a = W.CSR(m, n, rowptr, cc.astype(np.int32), dense[rr, cc].copy())
+    _, _, plan = run_and_compare(B, a, 0)
+    _, classes = B.spsyrk_plan_stats(plan)
+    assert sum(classes[6:]) >= m // 2
+    run_and_compare(B, a, 1)
