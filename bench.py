@@ -482,8 +482,7 @@ def run_ours(args):
             # ---- the accumulating form: C_L = tril(A_0 A_0^T) + tril(A_1 A_1^T) over two column panels of A
             if nnz_c * (4 + sv) < 20e9:
                 pt = []
-                for it in range(3):
-                    torch.cuda.empty_cache()
+                for it in range(3):  # the first round also warms the allocator: later rounds reuse its blocks
                     e = [ev()]
                     prods = []
                     for k0, k1 in ((0, a.n // 2), (a.n // 2, a.n)):
