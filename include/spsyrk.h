@@ -74,7 +74,7 @@ typedef enum { SPSYRK_TRIL = 0, SPSYRK_FULL = 1 } spsyrk_mode_t;
  * Row tiles: plans for disjoint row ranges are independent; concatenating their results gives
  * the untiled C_L.  (Halving a CSR matrix along rows is free, Section IV-A.)
  *
- * d_rowptr[m+1], d_colidx[nnz] (16-byte aligned), d_vals[nnz] of `dtype`.  0 <= row_begin <= row_end <= m.
+ * d_rowptr[m+1], d_colidx[nnz], d_vals[nnz] of `dtype`.  0 <= row_begin <= row_end <= m.
  * Errors: INVALID_ARG, OVERFLOW, WORKSPACE, BAD_CSR, CUDA.
  */
 spsyrk_status_t spsyrk_plan(spsyrk_plan_t *plan, int64_t m, int64_t n, int64_t nnz,
@@ -210,7 +210,7 @@ spsyrk_status_t spsyrk_accumulate(int64_t m, spsyrk_dtype_t dtype,
  *   1. d_workspace == NULL: *workspace_bytes receives the scratch size for (m, n, nnz, dtype).
  *   2. all pointers set: writes d_b_rowptr[m + 1], d_b_colidx[nnz], d_b_vals[nnz] (synchronises).
  * All pointers are device pointers except workspace_bytes (host); d_rperm has m entries, d_cperm n;
- * d_vals must be 16-byte aligned; B must not alias A.  Errors: INVALID_ARG (also: a map that is
+ * B must not alias A.  Errors: INVALID_ARG (also: a map that is
  * not a permutation), WORKSPACE, OVERFLOW, BAD_CSR (row pointers or column ids out of range), CUDA.
  */
 spsyrk_status_t spsyrk_permute(int64_t m, int64_t n, int64_t nnz, spsyrk_dtype_t dtype,

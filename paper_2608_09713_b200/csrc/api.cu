@@ -409,7 +409,6 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     if (!plan || !d_rowptr || (nnz > 0 && (!d_colidx || !d_vals))) return SPSYRK_ERR_INVALID_ARG;
     if (*workspace_bytes < need) return SPSYRK_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(d_workspace) % ALIGN) return SPSYRK_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(d_colidx) % 16) return SPSYRK_ERR_INVALID_ARG;  // tiles of it are copied 16 bytes at a time
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     spsyrk_plan_s* pl = new (std::nothrow) spsyrk_plan_s();

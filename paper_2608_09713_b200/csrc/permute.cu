@@ -175,7 +175,6 @@ extern "C" spsyrk_status_t spsyrk_permute(int64_t m, int64_t n, int64_t nnz, sps
     if (reinterpret_cast<uintptr_t>(d_workspace) % ALIGN) return SPSYRK_ERR_INVALID_ARG;
     if (!d_rowptr || !d_b_rowptr || (m > 0 && !d_rperm)) return SPSYRK_ERR_INVALID_ARG;
     if (nnz > 0 && (!d_colidx || !d_vals || !d_b_colidx || !d_b_vals)) return SPSYRK_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(d_vals) % 16) return SPSYRK_ERR_INVALID_ARG;  // tiles of it are copied 16 bytes at a time
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     PermuteWs w;
     carve(&w, d_workspace, m, n, nnz, sv);

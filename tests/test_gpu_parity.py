@@ -333,11 +333,20 @@ def test_workspace_and_alignment_errors(B):
     st = B._lib.spsyrk_plan(ctypes.byref(h), a.m, a.n, a.nnz, B._p(rowptr), B._p(colidx), B._p(vals), 0, 0, 0, a.m,
                             ctypes.c_void_p(ws.data_ptr() + 8), ctypes.byref(sz), None)
     assert st == 1                                                      # misaligned workspace
-    shifted = torch.empty(a.nnz + 1, dtype=torch.int32, device="cuda")
-    shifted[1:] = colidx
-    st = B._lib.spsyrk_plan(ctypes.byref(h), a.m, a.n, a.nnz, B._p(rowptr), ctypes.c_void_p(shifted.data_ptr() + 4),
-                            B._p(vals), 0, 0, 0, a.m, B._p(ws), ctypes.byref(sz), None)
-    assert st == 1                                                      # column ids not 16-byte aligned
+    # inputs need no particular alignment: column ids and values that start 4 / 8 bytes into an allocation
+    sc = torch.empty(a.nnz + 1, dtype=torch.int32, device="cuda")
+    sc[1:] = colidx
+    sv_ = torch.empty(a.nnz + 1, dtype=vals.dtype, device="cuda")
+    sv_[1:] = vals
+    rp2, ci2, cv2, _ = B.tril_syrk(a.m, a.n, rowptr, sc[1:], sv_[1:])
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL)
+    assert np.array_equal(rp2.cpu().numpy(), ref.rowptr) and np.array_equal(ci2.cpu().numpy(), ref.colidx)
+    check_values(cv2.cpu().numpy(), ref, a.vals.dtype)
+    sl = torch.empty(ci2.numel() + 1, dtype=torch.int32, device="cuda")
+    sl[1:] = ci2
+    f = B.spsyrk_mirror(a.m, rp2, sl[1:], cv2)
+    g = B.spsyrk_mirror(a.m, rp2, ci2, cv2)
+    assert all(torch.equal(x, y) for x, y in zip(f, g))
 
 
 # ---------------------------------------------------------------- blocks C[R, S] (Algorithm 2, lines 4 and 6)
