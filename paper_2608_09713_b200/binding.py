@@ -118,7 +118,8 @@ class Plan:
         return self.row_end - self.row_begin
 
     def close(self):
-        if self._h is not None:
+        # at interpreter shutdown the module's globals may already be gone: the process exit frees the plan
+        if self._h is not None and _lib is not None:
             _lib.spsyrk_destroy(self._h)
             self._h = None
 
