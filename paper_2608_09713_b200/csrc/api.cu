@@ -66,6 +66,7 @@ struct spsyrk_plan_s {
     uint32_t* colcnt;
     // radix sort buffers of the transpose (nnz entries each) and its histograms
     uint32_t *rx_key_a, *rx_row_a, *rx_pos_a, *rx_key_b, *rx_row_b, *rx_pos_b;
+    void *rx_val_a, *rx_val_b;
     uint32_t* rx_hist;
     int64_t* rx_offsets;
     int32_t* blockhist;
@@ -114,6 +115,8 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     auto rx_key_b = c.take<uint32_t>(nnz);
     auto rx_row_b = c.take<uint32_t>(nnz);
     auto rx_pos_b = c.take<uint32_t>(nnz);
+    auto rx_val_a = c.take<char>(nnz * sv);
+    auto rx_val_b = c.take<char>(nnz * sv);
     auto rx_hist = c.take<uint32_t>(rx_hist_n);
     auto rx_offsets = c.take<int64_t>(rx_hist_n + 1);
     auto blockhist = c.take<int32_t>(NCLASS * nb);
@@ -136,7 +139,7 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
         pl->desc_full = desc; pl->desc_blk = desc_blk;
         pl->perm = perm; pl->hdr = hdr; pl->cnt = cnt; pl->cls = cls; pl->colcnt = colcnt;
         pl->rx_key_a = rx_key_a; pl->rx_row_a = rx_row_a; pl->rx_pos_a = rx_pos_a; pl->rx_key_b = rx_key_b; pl->rx_row_b = rx_row_b;
-        pl->rx_pos_b = rx_pos_b; pl->rx_hist = rx_hist; pl->rx_offsets = rx_offsets;
+        pl->rx_pos_b = rx_pos_b; pl->rx_val_a = rx_val_a; pl->rx_val_b = rx_val_b; pl->rx_hist = rx_hist; pl->rx_offsets = rx_offsets;
         pl->blockhist = blockhist; pl->offsets = offsets; pl->partials = partials;
         pl->class_start_dev = class_start_dev; pl->work_total_dev = work_total_dev;
     }
@@ -181,8 +184,9 @@ int group_width(int64_t nnz, int64_t m) {
     return avg <= 4 ? 4 : avg <= 8 ? 8 : avg <= 16 ? 16 : 32;
 }
 
-// stable radix sort of the nonzeros by column id; the last pass writes the column lists and descriptors
-template <typename V>
+// stable radix sort of the nonzeros by column id; the last pass writes the column lists and descriptors.
+// VB: unsigned integer of the value's width (values are only moved)
+template <typename VB>
 spsyrk_status_t sort_by_column(spsyrk_plan_s* pl, cudaStream_t st) {
     constexpr int BITS = TRANSPOSE_RADIX_BITS;
     const PlanDev& P = pl->dev;
@@ -190,23 +194,26 @@ spsyrk_status_t sort_by_column(spsyrk_plan_s* pl, cudaStream_t st) {
     const int npass = (bits_for((uint64_t)std::max<int64_t>(P.n - 1, 1)) + BITS - 1) / BITS;
     const uint32_t* src_key = reinterpret_cast<const uint32_t*>(P.colidx);
     const uint32_t* src_row = pl->rx_row_b;
+    const VB* src_val = static_cast<const VB*>(P.vals);
     const uint32_t* src_pos = nullptr;  // position in A: the element's own index in the first pass
     for (int p = 0; p < npass; ++p) {
         const bool to_a = (p % 2) == 0;
         uint32_t* dst_key = to_a ? pl->rx_key_a : pl->rx_key_b;
         uint32_t* dst_row = to_a ? pl->rx_row_a : pl->rx_row_b;
         uint32_t* dst_pos = to_a ? pl->rx_pos_a : pl->rx_pos_b;
+        VB* dst_val = static_cast<VB*>(to_a ? pl->rx_val_a : pl->rx_val_b);
         if (p == npass - 1) {
-            EmitTransposeFinal<V> emit{P};
-            SPSYRK_CUDA_TRY((radix_pass<BITS, uint32_t>(src_key, src_row, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
-                                                        pl->partials, emit, st)));
+            EmitTransposeFinal<VB> emit{P};
+            SPSYRK_CUDA_TRY((radix_pass3<BITS, VB>(src_key, src_row, src_val, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
+                                                   pl->partials, emit, st)));
         } else {
-            EmitArrays<uint32_t> emit{dst_key, dst_row, dst_pos};
-            SPSYRK_CUDA_TRY((radix_pass<BITS, uint32_t>(src_key, src_row, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
-                                                        pl->partials, emit, st)));
+            EmitArrays3<VB> emit{dst_key, dst_row, dst_val, dst_pos};
+            SPSYRK_CUDA_TRY((radix_pass3<BITS, VB>(src_key, src_row, src_val, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
+                                                   pl->partials, emit, st)));
         }
         src_key = dst_key;
         src_row = dst_row;
+        src_val = dst_val;
         src_pos = dst_pos;
     }
     return SPSYRK_OK;

@@ -62,11 +62,12 @@ struct emit_wants_neighbours : std::false_type {};
 template <typename E>
 struct emit_wants_neighbours<E, std::void_t<decltype(E::NEIGHBOURS)>> : std::bool_constant<E::NEIGHBOURS> {};
 
-template <int BITS, typename PB>
+template <int BITS, typename PB, bool HAS_PC = false>
 struct RadixSmem {
     static constexpr int NB = 1 << BITS;
     static size_t bytes() {
-        return (size_t)NB * 8 + (size_t)RX_TILE * sizeof(PB) + (size_t)RX_TILE * (4 + 4) + (size_t)RX_WARPS * NB * 4 + (size_t)NB * 4;
+        return (size_t)NB * 8 + (size_t)RX_TILE * sizeof(PB) + (size_t)RX_TILE * (4 + 4 + (HAS_PC ? 4 : 0)) + (size_t)RX_WARPS * NB * 4 +
+               (size_t)NB * 4;
     }
 };
 
@@ -78,10 +79,13 @@ struct RadixSmem {
 // the payloads still in flight while the keys are ranked), learns each element's slot in the tile's
 // digit-major order, drops key and payloads into that slot of shared memory, and the tile is then
 // read back slot by slot and written out in runs.
-template <int BITS, typename PB, typename Emit>
+// HAS_PC: a third payload pc (32 bits; nullptr = the element's own index) travels along and the functor is
+// called as emit(dest, key, pa, pb, pc).
+template <int BITS, typename PB, typename Emit, bool HAS_PC = false>
 __global__ void __launch_bounds__(RX_THREADS, 2) radix_scatter_kernel(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pa,
-                                                                      const PB* __restrict__ pb, int64_t n, int shift,
-                                                                      const int64_t* __restrict__ goff_all, int64_t ntiles, Emit emit) {
+                                                                      const PB* __restrict__ pb, const uint32_t* __restrict__ pc,
+                                                                      int64_t n, int shift, const int64_t* __restrict__ goff_all,
+                                                                      int64_t ntiles, Emit emit) {
     constexpr int NB = 1 << BITS;
     static_assert(BITS <= 12, "digit width");
     extern __shared__ __align__(16) unsigned char rx_smem[];
@@ -90,7 +94,8 @@ __global__ void __launch_bounds__(RX_THREADS, 2) radix_scatter_kernel(const uint
     PB* s_pb = reinterpret_cast<PB*>(goff + NB);                       // [TILE] sorted order
     uint32_t* s_key = reinterpret_cast<uint32_t*>(s_pb + RX_TILE);     // [TILE] sorted order
     uint32_t* s_pa = s_key + RX_TILE;                                  // [TILE] sorted order
-    uint32_t* wcount = s_pa + RX_TILE;                                 // [WARPS][NB]
+    uint32_t* s_pc = s_pa + RX_TILE;                                   // [TILE] sorted order (HAS_PC only)
+    uint32_t* wcount = s_pc + (HAS_PC ? RX_TILE : 0);                  // [WARPS][NB]
     uint32_t* bin_start = wcount + RX_WARPS * NB;                      // [NB]
 
     const int tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
@@ -185,13 +190,17 @@ __global__ void __launch_bounds__(RX_THREADS, 2) radix_scatter_kernel(const uint
             s_key[q] = k[i];
             s_pa[q] = a[i];
             s_pb[q] = b[i];
+            // the third payload is loaded only now: it would not fit the registers next to the others
+            if constexpr (HAS_PC) s_pc[q] = pc ? pc[tile_base + t] : (uint32_t)(tile_base + t);
         }
     }
     __syncthreads();
     for (int q = tid; q < tile_n; q += RX_THREADS) {
         const uint32_t key = s_key[q];
         const int64_t dest = goff[(key >> shift) & (NB - 1)] + q;
-        if constexpr (emit_wants_neighbours<Emit>::value) {
+        if constexpr (HAS_PC) {
+            emit(dest, key, s_pa[q], s_pb[q], s_pc[q]);
+        } else if constexpr (emit_wants_neighbours<Emit>::value) {
             // the keys of the slots before and after (NO_KEY at the ends of the tile): in the last pass of a
             // sort equal keys are adjacent, so a functor can tell where a run of one key starts and ends
             emit(dest, key, s_pa[q], s_pb[q], q > 0 ? s_key[q - 1] : NO_KEY, q + 1 < tile_n ? s_key[q + 1] : NO_KEY);
@@ -213,23 +222,50 @@ struct EmitArrays {
     }
 };
 
+template <typename PB>
+struct EmitArrays3 {
+    uint32_t* keys;
+    uint32_t* pa;
+    PB* pb;
+    uint32_t* pc;
+    __device__ __forceinline__ void operator()(int64_t dest, uint32_t k, uint32_t a, PB b, uint32_t c) const {
+        keys[dest] = k;
+        pa[dest] = a;
+        pb[dest] = b;
+        pc[dest] = c;
+    }
+};
+
 // hist: NB * ntiles uint32; offsets: NB * ntiles + 1 int64; partials: scan_partials_count(NB * ntiles) int64
-template <int BITS, typename PB, typename Emit>
-inline cudaError_t radix_pass(const uint32_t* keys, const uint32_t* pa, const PB* pb, int64_t n, int shift, uint32_t* hist,
-                              int64_t* offsets, int64_t* partials, Emit emit, cudaStream_t st) {
+template <int BITS, typename PB, bool HAS_PC, typename Emit>
+inline cudaError_t radix_pass_impl(const uint32_t* keys, const uint32_t* pa, const PB* pb, const uint32_t* pc, int64_t n, int shift,
+                                   uint32_t* hist, int64_t* offsets, int64_t* partials, Emit emit, cudaStream_t st) {
     constexpr int NB = 1 << BITS;
     const int64_t nt = radix_tiles(n);
     if (nt == 0) return cudaSuccess;
     radix_hist_kernel<BITS><<<(unsigned)nt, RX_THREADS, 0, st>>>(keys, n, shift, hist, nt);
     cudaError_t e = exclusive_scan_i64<uint32_t>(hist, (int64_t)NB * nt, offsets, partials, st);
     if (e != cudaSuccess) return e;
-    auto kern = radix_scatter_kernel<BITS, PB, Emit>;
-    const size_t smem = RadixSmem<BITS, PB>::bytes();
+    auto kern = radix_scatter_kernel<BITS, PB, Emit, HAS_PC>;
+    const size_t smem = RadixSmem<BITS, PB, HAS_PC>::bytes();
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<(unsigned)nt, RX_THREADS, smem, st>>>(keys, pa, pb, n, shift, offsets, nt, emit);
+    kern<<<(unsigned)nt, RX_THREADS, smem, st>>>(keys, pa, pb, pc, n, shift, offsets, nt, emit);
     note_launches(2);
     return cudaGetLastError();
+}
+
+template <int BITS, typename PB, typename Emit>
+inline cudaError_t radix_pass(const uint32_t* keys, const uint32_t* pa, const PB* pb, int64_t n, int shift, uint32_t* hist,
+                              int64_t* offsets, int64_t* partials, Emit emit, cudaStream_t st) {
+    return radix_pass_impl<BITS, PB, false>(keys, pa, pb, nullptr, n, shift, hist, offsets, partials, emit, st);
+}
+
+// the same with a third 32-bit payload (pc == nullptr: the element's own index)
+template <int BITS, typename PB, typename Emit>
+inline cudaError_t radix_pass3(const uint32_t* keys, const uint32_t* pa, const PB* pb, const uint32_t* pc, int64_t n, int shift,
+                               uint32_t* hist, int64_t* offsets, int64_t* partials, Emit emit, cudaStream_t st) {
+    return radix_pass_impl<BITS, PB, true>(keys, pa, pb, pc, n, shift, hist, offsets, partials, emit, st);
 }
 
 inline int bits_for(uint64_t max_value) {

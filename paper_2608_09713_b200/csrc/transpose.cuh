@@ -8,9 +8,11 @@
 //             column length (FULL).  "Rows j <= i of column k" is then at_row[start, start+len).
 //
 // Method: histogram of column ids and scan for colptr; then a stable LSD radix sort of the
-// nonzeros by column id with (row, position in A) as payload.  The nonzeros enter in row order, so
-// each column's segment comes out ascending by row; the last pass writes at_row, gathers the
-// value and scatters the descriptor, whose length is the entry's rank inside its column.
+// nonzeros by column id with (row, value, position in A) as payload.  The nonzeros enter in row
+// order, so each column's segment comes out ascending by row; the last pass writes at_row and
+// at_val and scatters the descriptor, whose length is the entry's rank inside its column.  (The
+// value travels with the element because reading it in the first pass is sequential, whereas
+// fetching it by position in the last pass is one random access per nonzero.)
 #pragma once
 #include "radix.cuh"
 
@@ -68,13 +70,13 @@ static __global__ void __launch_bounds__(256) row_expand_kernel(const int64_t* _
 }
 
 // last radix pass of the transpose: the element at sorted position s is entry s of the column lists
-template <typename V>
+template <typename VB>
 struct EmitTransposeFinal {
     PlanDev P;
-    __device__ __forceinline__ void operator()(int64_t s, uint32_t k, uint32_t row, uint32_t p) const {
+    __device__ __forceinline__ void operator()(int64_t s, uint32_t k, uint32_t row, VB val, uint32_t p) const {
         const int64_t cs = P.colptr[k];
         P.at_row[s] = (int32_t)row;
-        static_cast<V*>(P.at_val)[s] = static_cast<const V*>(P.vals)[p];
+        static_cast<VB*>(P.at_val)[s] = val;  // bit copy of the value that travelled with the element
         P.desc[p] = make_uint2((uint32_t)cs, P.mode == SPSYRK_TRIL ? (uint32_t)(s - cs) + 1u : (uint32_t)(P.colptr[k + 1] - cs));
     }
 };
