@@ -175,7 +175,8 @@ template <int G>
 void launch_row_work(spsyrk_plan_s* pl, cudaStream_t st) {
     const PlanDev& P = pl->dev;
     const int64_t threads = (int64_t)(P.r1 - P.r0) * G;
-    row_work_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P, pl->cls, BLOCK_CLASS_MAX_WORK, pl->work_total_dev);
+    const int64_t ctas = std::min<int64_t>((threads + 255) / 256, (int64_t)pl->sm_count * 16);
+    row_work_kernel<G><<<(unsigned)ctas, 256, 0, st>>>(P, pl->cls, BLOCK_CLASS_MAX_WORK, pl->work_total_dev);
     note_launches(1);
 }
 

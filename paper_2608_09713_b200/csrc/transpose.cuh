@@ -108,32 +108,36 @@ static __global__ void __launch_bounds__(256) block_desc_kernel(PlanDev P, const
 template <int G>
 static __global__ void __launch_bounds__(256) row_work_kernel(PlanDev P, uint8_t* __restrict__ cls, int64_t block_max,
                                                         unsigned long long* __restrict__ work_total) {
-    const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
     const int gl = threadIdx.x & (G - 1);
     const int64_t rows = P.r1 - P.r0;
-    int64_t w = 0, deg = 0;
-    if (gid < rows) {
-        const int64_t i = P.r0 + gid;
-        const int64_t p0 = P.rowptr[i], p1 = P.rowptr[i + 1];
-        deg = p1 - p0;
-        for (int64_t p = p0 + gl; p < p1; p += G) w += P.desc[p].y;
-    }
+    const int64_t groups = ((int64_t)gridDim.x * blockDim.x) / G;
+    unsigned long long mine = 0;  // work of the rows this thread owned
+    // a fixed grid walks the rows: one atomic per CTA for the total, however many rows there are
+    for (int64_t gbase = ((int64_t)blockIdx.x * blockDim.x) / G; gbase < rows; gbase += groups) {  // uniform per CTA
+        const int64_t gid = gbase + threadIdx.x / G;
+        int64_t w = 0, deg = 0;
+        if (gid < rows) {
+            const int64_t i = P.r0 + gid;
+            const int64_t p0 = P.rowptr[i], p1 = P.rowptr[i + 1];
+            deg = p1 - p0;
+            for (int64_t p = p0 + gl; p < p1; p += G) w += P.desc[p].y;
+        }
 #pragma unroll
-    for (int o = G / 2; o > 0; o >>= 1) w += __shfl_xor_sync(FULL_MASK, w, o);
-    const bool owner = gid < rows && gl == 0;
-    if (owner) {
-        P.work[gid] = w;
-        uint8_t c;
-        if (w == 0) c = 0;
-        else if (deg <= 32 && w <= 512) c = w <= 32 ? 1 : w <= 64 ? 2 : w <= 128 ? 3 : w <= 256 ? 4 : 5;
-        else c = w <= block_max ? 6 : 7;
-        cls[gid] = c;
+        for (int o = G / 2; o > 0; o >>= 1) w += __shfl_xor_sync(FULL_MASK, w, o);
+        if (gid < rows && gl == 0) {
+            P.work[gid] = w;
+            uint8_t c;
+            if (w == 0) c = 0;
+            else if (deg <= 32 && w <= 512) c = w <= 32 ? 1 : w <= 64 ? 2 : w <= 128 ? 3 : w <= 256 ? 4 : 5;
+            else c = w <= block_max ? 6 : 7;
+            cls[gid] = c;
+            mine += (unsigned long long)w;
+        }
     }
-    // one atomic per CTA for the total
     __shared__ unsigned long long cta_sum;
     if (threadIdx.x == 0) cta_sum = 0;
     __syncthreads();
-    unsigned long long ws = warp_reduce_sum<unsigned long long>(owner ? (unsigned long long)w : 0ull);
+    const unsigned long long ws = warp_reduce_sum<unsigned long long>(mine);
     if (lane_id() == 0 && ws) atomicAdd(&cta_sum, ws);
     __syncthreads();
     if (threadIdx.x == 0 && cta_sum) atomicAdd(work_total, cta_sum);
