@@ -104,13 +104,20 @@ __global__ void mirror_rowtot_kernel(const int64_t* __restrict__ l_rowptr, const
 __global__ void mirror_last_entry_kernel(const int64_t* __restrict__ l_rowptr, const int32_t* __restrict__ l_colidx, int64_t m,
                                          uint32_t* err) {
     const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= m) return;
-    const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
-    if (p1 < p0) { atomicOr(err, ERRW_BAD_ROWPTR); return; }
-    if (p1 == p0) return;
-    const int64_t last = l_colidx[p1 - 1], first = l_colidx[p0];
-    if (last > r || first < 0) atomicOr(err, ERRW_UPPER);
-    else if (last == r) atomicAdd(err + 1, 1u);
+    bool diag = false;
+    if (r < m) {
+        const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
+        if (p1 < p0) {
+            atomicOr(err, ERRW_BAD_ROWPTR);
+        } else if (p1 > p0) {
+            const int64_t last = l_colidx[p1 - 1], first = l_colidx[p0];
+            if (last > r || first < 0) atomicOr(err, ERRW_UPPER);
+            else diag = last == r;
+        }
+    }
+    // one atomic per warp: nearly every row of a product stores its diagonal
+    const unsigned votes = __ballot_sync(FULL_MASK, diag);
+    if (lane_id() == 0 && votes) atomicAdd(err + 1, (uint32_t)__popc(votes));
 }
 
 // G lanes per row: the explicit (key, row) pair of every entry
