@@ -119,7 +119,7 @@ def whole_job_rate(units_per_rank: float, world: int, ms_per_step: float) -> flo
 def class_of_rows(work, deg):
     """The library's row classes, recomputed on the host for the roofline's byte counts."""
     cls = np.full(work.shape, 7, dtype=np.int8)
-    cls[work <= 16384] = 6
+    cls[work <= 8192] = 6
     light = (deg <= 32) & (work <= 512)
     for c, hi in ((5, 512), (4, 256), (3, 128), (2, 64), (1, 32)):
         cls[light & (work <= hi)] = c

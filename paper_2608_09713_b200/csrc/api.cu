@@ -19,7 +19,7 @@ void note_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); 
 namespace {
 
 constexpr size_t ALIGN = 256;
-constexpr int64_t BLOCK_CLASS_MAX_WORK = 16384;  // class 6 (256-thread CTA) up to here, class 7 above
+constexpr int64_t BLOCK_CLASS_MAX_WORK = 8192;  // class 6 (256-thread CTA) up to here, class 7 above
 constexpr uint32_t ROW_CHUNK_BITS_MAX_NUMERIC = 1u << 18;
 constexpr uint32_t ROW_CHUNK_BITS_MAX_SYMBOLIC = 1u << 20;
 constexpr int TRANSPOSE_RADIX_BITS = 8;

@@ -596,7 +596,7 @@ def test_plan_partition(B, idx):
 # ------------------------------------------------------------------ rows exactly at the class boundaries
 def test_rows_at_every_class_boundary(B):
     """One column shared by all rows: row i has exactly i + 1 partial products and i + 1 output entries,
-    so consecutive rows walk through every class boundary (32|33, 64|65, ..., 512|513, 16384|16385).
+    so consecutive rows walk through every class boundary (32|33, 64|65, ..., 512|513, 8192|8193).
     Structure by closed form for every row, values (single products, exact) for every entry, and rows
     around the boundaries against the oracle."""
     m = 16500
@@ -608,13 +608,13 @@ def test_rows_at_every_class_boundary(B):
     assert np.array_equal(rp.cpu().numpy(), i * (i + 1) // 2)
     work, classes = B.spsyrk_plan_stats(plan)
     assert work == m * (m + 1) // 2
-    assert classes == [0, 32, 32, 64, 128, 256, 16384 - 512, m - 16384]
+    assert classes == [0, 32, 32, 64, 128, 256, 8192 - 512, m - 8192]
     rows = torch.repeat_interleave(torch.arange(m, device="cuda"), torch.arange(1, m + 1, device="cuda"))
     cols = torch.arange(ci.numel(), device="cuda") - rp[:-1][rows]
     assert torch.equal(ci.long(), cols)
     v = torch.from_numpy(vals).cuda()
     assert torch.equal(cv, v[rows] * v[cols])                 # one product per entry: no rounding to differ in
-    for r in (0, 31, 32, 63, 64, 127, 128, 255, 256, 511, 512, 16383, 16384, m - 1):
+    for r in (0, 31, 32, 63, 64, 127, 128, 255, 256, 511, 512, 8191, 8192, m - 1):
         ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, r, r + 1)
         lo, hi = int(rp[r]), int(rp[r + 1])
         assert np.array_equal(ci[lo:hi].cpu().numpy(), ref.colidx)
