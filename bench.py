@@ -251,6 +251,10 @@ def run_ours(args):
                     torch.empty(nnz_f0, dtype=d_vals.dtype, device="cuda"))
     if is_int:
         buf["jac"] = torch.empty(max(nnz0, 1), dtype=torch.float32, device="cuda")
+    if not args.no_map:
+        p0 = B.spsyrk_plan(a.m, a.n, d_rowptr, d_colidx, d_vals, mode=B.TRIL, row_begin=r0, row_end=r1, workspace=buf["plan_ws"])
+        buf["map"] = torch.empty(max(B.spsyrk_plan_map_bytes(p0), 256), dtype=torch.uint8, device="cuda")
+        del p0
 
     def step(timing=False, keep=False):
         marks = [ev()]
@@ -259,6 +263,8 @@ def run_ours(args):
             B.spsyrk_plan_enable_timing(plan)
         if shard:
             B.spsyrk_plan_set_rows(plan, *S.rank_rows(B.spsyrk_plan_partition(plan, world), rank))
+        if "map" in buf:
+            B.spsyrk_plan_lend_map(plan, buf["map"])
         marks.append(ev())
         c_rowptr, c_colidx, c_vals = buf["c_rowptr"], buf["c_colidx"], buf["c_vals"]
         nnz = B.spsyrk_symbolic(plan, c_rowptr)
@@ -547,6 +553,7 @@ def main():
     ap.add_argument("--workload", type=int, default=5, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--no-mirror", action="store_true")
     ap.add_argument("--no-full", action="store_true")
+    ap.add_argument("--no-map", action="store_true", help="do not lend the item map: symbolic counts with hash sets, numeric sorts")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--rmat-noperm", action="store_true", help="with --rmat-scale: skip the random relabelling (load-balance study)")
     ap.add_argument("--shard-rows", action="store_true",

@@ -109,6 +109,28 @@ spsyrk_status_t spsyrk_plan_set_block(spsyrk_plan_t plan, int64_t row_begin, int
                                       int64_t col_begin, int64_t col_end, void *cuda_stream);
 
 /*
+ * spsyrk_plan_map_bytes / spsyrk_plan_lend_map - optional item map for the light rows.
+ *
+ * A light row (at most 32 nonzeros, at most 512 partial products) is computed from the list of its
+ * partial products a_ik * a_jk, "items", in ascending k and j.  Producing the row sorted by j means
+ * ordering the items by j; that ordering depends on the structure of A only.  If the caller lends a
+ * device buffer of spsyrk_plan_map_bytes bytes (two bytes per item of the plan's current row range,
+ * rows padded to eight items), spsyrk_symbolic orders the items once and records for every item the
+ * output slot it adds into and its place among the items of that slot, and spsyrk_numeric only
+ * gathers, multiplies and adds - also for every later spsyrk_numeric call on the same structure.
+ * Without a map (or with one that is too small for the current row range) symbolic counts with a
+ * hash set and numeric sorts by itself; the results are identical bit for bit either way
+ * (both add the partial products of an entry in ascending k: Section II-A's dot product, left to right).
+ *
+ * The size is known after spsyrk_plan / spsyrk_plan_set_rows / spsyrk_plan_set_block (it changes with
+ * the row range).  The buffer is caller-owned, 256-byte aligned, and must stay valid from
+ * spsyrk_symbolic to the last spsyrk_numeric that uses it; lending invalidates any symbolic result.
+ * d_map == NULL takes the map back.  Errors: INVALID_ARG.
+ */
+spsyrk_status_t spsyrk_plan_map_bytes(spsyrk_plan_t plan, size_t *bytes);
+spsyrk_status_t spsyrk_plan_lend_map(spsyrk_plan_t plan, void *d_map, size_t bytes);
+
+/*
  * spsyrk_symbolic - count the stored entries of every output row of the plan's range and
  * turn the counts into row pointers.
  *   cnt[i] = #{ j <= i : rows i and j of A share a column }   (TRIL; all j in FULL mode)

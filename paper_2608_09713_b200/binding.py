@@ -39,6 +39,10 @@ _lib.spsyrk_plan_set_rows.argtypes = [_vp, _i64, _i64, _vp]
 _lib.spsyrk_plan_set_block.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp]
 _lib.spsyrk_plan_set_block.restype = _int
 _lib.spsyrk_symbolic.argtypes = [_vp, _vp, _i64p, _vp]
+_lib.spsyrk_plan_map_bytes.argtypes = [_vp, _szp]
+_lib.spsyrk_plan_map_bytes.restype = _int
+_lib.spsyrk_plan_lend_map.argtypes = [_vp, _vp, ctypes.c_size_t]
+_lib.spsyrk_plan_lend_map.restype = _int
 _lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_column_panel.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
@@ -162,6 +166,22 @@ def spsyrk_plan_set_block(plan: Plan, row_begin: int, row_end: int, col_begin: i
     _check(_lib.spsyrk_plan_set_block(plan._h, row_begin, row_end, col_begin, col_end, _stream(stream)),
            "spsyrk_plan_set_block")
     plan.row_begin, plan.row_end = row_begin, row_end
+
+
+def spsyrk_plan_map_bytes(plan: Plan) -> int:
+    sz = ctypes.c_size_t(0)
+    _check(_lib.spsyrk_plan_map_bytes(plan._h, ctypes.byref(sz)), "spsyrk_plan_map_bytes")
+    return sz.value
+
+
+def spsyrk_plan_lend_map(plan: Plan, item_map: torch.Tensor | None):
+    """Lend (or, with None, take back) the item map: a uint8 CUDA tensor of at least spsyrk_plan_map_bytes bytes."""
+    if item_map is not None:
+        _dev_check(item_map)
+        assert item_map.dtype == torch.uint8
+    _check(_lib.spsyrk_plan_lend_map(plan._h, _p(item_map), 0 if item_map is None else item_map.numel()),
+           "spsyrk_plan_lend_map")
+    plan._keep["map"] = item_map
 
 
 def spsyrk_symbolic(plan: Plan, c_rowptr: torch.Tensor, stream=None) -> int:
@@ -408,10 +428,15 @@ def spsyrk_host_release_cache():
 # ------------------------------------------------------------------------------------------
 # Convenience: the calls a user makes for one product, outputs allocated with torch.
 # ------------------------------------------------------------------------------------------
-def tril_syrk(m, n, rowptr, colidx, vals, mode=TRIL, row_begin=0, row_end=None, plan: Plan | None = None, stream=None):
-    """plan -> symbolic -> numeric.  Returns (c_rowptr, c_colidx, c_vals, plan)."""
+def tril_syrk(m, n, rowptr, colidx, vals, mode=TRIL, row_begin=0, row_end=None, plan: Plan | None = None, stream=None,
+              item_map=True):
+    """plan -> (item map) -> symbolic -> numeric.  Returns (c_rowptr, c_colidx, c_vals, plan)."""
     if plan is None:
         plan = spsyrk_plan(m, n, rowptr, colidx, vals, mode, row_begin, row_end, stream)
+    if item_map:
+        spsyrk_plan_lend_map(plan, _workspace(spsyrk_plan_map_bytes(plan), rowptr.device))
+    else:
+        spsyrk_plan_lend_map(plan, None)
     c_rowptr = torch.empty(plan.rows + 1, dtype=torch.int64, device=rowptr.device)
     nnz = spsyrk_symbolic(plan, c_rowptr, stream)
     c_colidx = torch.empty(max(nnz, 1), dtype=torch.int32, device=rowptr.device)

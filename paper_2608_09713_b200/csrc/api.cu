@@ -77,6 +77,11 @@ struct spsyrk_plan_s {
     uint32_t* row_counter;  // row dispenser of the persistent heavy-row kernel
     double* gacc;           // its global accumulator slices (GLOBAL_ACC_CTAS x gslots, 8 bytes per slot)
     uint32_t gslots;
+    int64_t* itemoff;      // rows + 1, class order: where the map words of a light row start
+    int64_t map_items;     // map words the current row range needs
+    uint16_t* map;         // caller's item map (spsyrk_plan_lend_map), or null
+    size_t map_bytes;
+    bool map_filled;       // the last symbolic pass wrote the map
     int64_t* work_prefix;  // rows + 1: exclusive prefix sums of the per-row work (spsyrk_plan_partition)
     int64_t* part_bounds;  // MAX_PARTS + 1
     // host facts
@@ -84,6 +89,7 @@ struct spsyrk_plan_s {
     int64_t work_total;
     bool have_symbolic;
     bool key64;
+    bool diag;  // the light-row kernels handle the diagonal apart (lower-triangle mode, whole column range)
     int sm_count;
     // optional per-class timing of the symbolic and numeric launches
     bool timing;
@@ -98,8 +104,9 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     const int64_t items = std::max<int64_t>(std::max(m, n), 1);
     const int64_t nb = bin_blocks(items);
     auto colptr = c.take<int64_t>(n + 1);
-    auto at_row = c.take<int32_t>(nnz);
+    auto at_row = c.take<int32_t>(nnz + 4);  // the symbolic gathers read aligned 16-byte pieces: up to 3 entries past the end
     auto at_val = c.take<char>(nnz * sv);
+    auto at_rec = c.take<char>(nnz * (sv == 8 ? 16 : 8));
     auto desc = c.take<uint2>(nnz);
     auto desc_blk = c.take<uint2>(nnz);
     auto work = c.take<int64_t>(m);
@@ -127,14 +134,15 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     auto err = c.take<uint32_t>(1);
     auto row_counter = c.take<uint32_t>(1);
     auto work_prefix = c.take<int64_t>(items + 1);
+    auto itemoff = c.take<int64_t>(items + 1);
     auto part_bounds = c.take<int64_t>(MAX_PARTS + 1);
     // one global accumulator slice per persistent CTA of the heavy-row numeric kernel
     const uint32_t gslots = pow2_at_least((uint64_t)std::max<int64_t>(m, 1), 1024u, ROW_CHUNK_BITS_MAX_NUMERIC);
     auto gacc = c.take<double>((size_t)GLOBAL_ACC_CTAS * gslots);
     if (pl) {
         pl->row_counter = row_counter; pl->gacc = gacc; pl->gslots = gslots;
-        pl->work_prefix = work_prefix; pl->part_bounds = part_bounds;
-        pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.desc = desc;
+        pl->work_prefix = work_prefix; pl->part_bounds = part_bounds; pl->itemoff = itemoff;
+        pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.at_rec = at_rec; pl->dev.desc = desc;
         pl->dev.work = work; pl->dev.err = err;
         pl->desc_full = desc; pl->desc_blk = desc_blk;
         pl->perm = perm; pl->hdr = hdr; pl->cnt = cnt; pl->cls = cls; pl->colcnt = colcnt;
@@ -176,7 +184,7 @@ void launch_row_work(spsyrk_plan_s* pl, cudaStream_t st) {
     const PlanDev& P = pl->dev;
     const int64_t threads = (int64_t)(P.r1 - P.r0) * G;
     const int64_t ctas = std::min<int64_t>((threads + 255) / 256, (int64_t)pl->sm_count * 16);
-    row_work_kernel<G><<<(unsigned)ctas, 256, 0, st>>>(P, pl->cls, BLOCK_CLASS_MAX_WORK, pl->work_total_dev);
+    row_work_kernel<G><<<(unsigned)ctas, 256, 0, st>>>(P, pl->cls, BLOCK_CLASS_MAX_WORK, pl->diag, pl->work_total_dev);
     note_launches(1);
 }
 
@@ -239,6 +247,7 @@ spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
         }
     }
     const PlanDev& P = pl->dev;
+    pl->diag = P.mode == SPSYRK_TRIL && pl->dev.desc == pl->desc_full;
     SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->work_total_dev, 0, sizeof(unsigned long long), st));
     if (rows > 0) {
         switch (group_width(P.nnz, P.m)) {
@@ -253,47 +262,149 @@ spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
         row_header_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(P, pl->perm, rows, pl->hdr);
         note_launches(1);
     }
+    // where the item-map words of every light row start (rows in class order)
+    int64_t map_items = 0;
+    pl->map_filled = false;
+    if (rows > 0) {
+        uint32_t* items8 = reinterpret_cast<uint32_t*>(pl->cnt);  // free until the symbolic pass
+        row_items_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(P, pl->hdr, pl->cls, rows, pl->diag, items8);
+        note_launches(1);
+        SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(items8, rows, pl->itemoff, pl->partials, st));
+        SPSYRK_CUDA_TRY(cudaMemcpyAsync(&map_items, pl->itemoff + rows, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
+    }
     unsigned long long wt = 0;
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(pl->class_start, pl->class_start_dev, sizeof(pl->class_start), cudaMemcpyDeviceToHost, st));
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(&wt, pl->work_total_dev, sizeof(wt), cudaMemcpyDeviceToHost, st));
     spsyrk_status_t s = read_err(pl, st);
     pl->work_total = (int64_t)wt;
+    pl->map_items = map_items;
     return s;
 }
 
-template <int N>
-void launch_symbolic_warp(spsyrk_plan_s* pl, int c, cudaStream_t st) {
+bool use_map(const spsyrk_plan_s* pl) { return pl->map && pl->map_bytes >= (size_t)pl->map_items * sizeof(uint16_t); }
+
+template <int N, bool DIAG>
+spsyrk_status_t launch_symbolic_warp_d(spsyrk_plan_s* pl, int c, cudaStream_t st) {
     const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
-    if (count <= 0) return;
+    if (count <= 0) return SPSYRK_OK;
+    constexpr int G = warp_class_group(N);
     constexpr int SW = symbolic_warps(N);
-    auto kern = pl->dev.desc == pl->desc_blk ? symbolic_warp_kernel<N, true> : symbolic_warp_kernel<N, false>;
+    constexpr int ROWS = SW * (32 / G);  // rows a CTA works on at a time
+    constexpr size_t smem = (size_t)ROWS * SymbolicWarpSmem<N>::GROUP;
+    auto kern = symbolic_warp_kernel<N, G, DIAG>;
+    SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, SW * 32, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
-    const int64_t want = (count + SW - 1) / SW;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, SW * 32, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const int64_t want = (count + ROWS - 1) / ROWS;
     const int64_t cap = (int64_t)pl->sm_count * per_sm;
-    kern<<<(unsigned)std::min(want, cap), SW * 32, 0, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, pl->cnt);
+    kern<<<(unsigned)std::min(want, cap), SW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, pl->cnt);
     note_launches(1);
+    return SPSYRK_OK;
+}
+
+template <int N>
+spsyrk_status_t launch_symbolic_warp(spsyrk_plan_s* pl, int c, cudaStream_t st) {
+    return pl->diag ? launch_symbolic_warp_d<N, true>(pl, c, st) : launch_symbolic_warp_d<N, false>(pl, c, st);
+}
+
+template <typename V, int N, typename Key, bool DIAG>
+spsyrk_status_t launch_numeric_warp_d(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    if (count <= 0) return SPSYRK_OK;
+    constexpr int G = warp_class_group(N);
+    constexpr int NW = numeric_warps(N);
+    constexpr int ROWS = NW * (32 / G);
+    constexpr size_t smem = (size_t)ROWS * NumericWarpSmem<V, N>::GROUP;
+    // persistent groups: exactly as many CTAs as are resident at once, each group walks its rows with
+    // a stride of the whole grid
+    auto kern = numeric_warp_kernel<V, N, G, Key, DIAG>;
+    SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const int64_t want = (count + ROWS - 1) / ROWS;
+    const int64_t cap = (int64_t)pl->sm_count * per_sm;
+    kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, c_rowptr, c_colidx,
+                                                               static_cast<V*>(c_vals));
+    note_launches(1);
+    return SPSYRK_OK;
 }
 
 template <typename V, int N, typename Key>
-void launch_numeric_warp(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+spsyrk_status_t launch_numeric_warp(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    return pl->diag ? launch_numeric_warp_d<V, N, Key, true>(pl, c, c_rowptr, c_colidx, c_vals, st)
+                    : launch_numeric_warp_d<V, N, Key, false>(pl, c, c_rowptr, c_colidx, c_vals, st);
+}
+
+template <int N, typename Key, bool DIAG>
+spsyrk_status_t launch_symbolic_sort_d(spsyrk_plan_s* pl, int c, cudaStream_t st) {
     const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
-    if (count <= 0) return;
-    constexpr int NW = numeric_warps(N);
-    // persistent warps: exactly as many CTAs as are resident at once, each warp walks its rows with
-    // a stride of the whole grid
-    auto kern = pl->dev.desc == pl->desc_blk ? numeric_warp_kernel<V, N, Key, true> : numeric_warp_kernel<V, N, Key, false>;
+    if (count <= 0) return SPSYRK_OK;
+    constexpr int G = warp_class_group(N);
+    constexpr int SW = symbolic_sort_warps(N);
+    constexpr int ROWS = SW * (32 / G);
+    constexpr size_t smem = (size_t)ROWS * SymbolicSortSmem<N>::GROUP;
+    auto kern = symbolic_sort_warp_kernel<N, G, Key, DIAG>;
+    SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
-    const int64_t want = (count + NW - 1) / NW;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, SW * 32, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const int64_t want = (count + ROWS - 1) / ROWS;
     const int64_t cap = (int64_t)pl->sm_count * per_sm;
-    kern<<<(unsigned)std::min(want, cap), NW * 32, 0, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, c_rowptr, c_colidx,
-                                                            static_cast<V*>(c_vals));
+    kern<<<(unsigned)std::min(want, cap), SW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], pl->itemoff + pl->class_start[c],
+                                                               count, pl->cnt, pl->map);
     note_launches(1);
+    return SPSYRK_OK;
+}
+
+template <int N>
+spsyrk_status_t launch_symbolic_sort(spsyrk_plan_s* pl, int c, cudaStream_t st) {
+    if (pl->key64)
+        return pl->diag ? launch_symbolic_sort_d<N, uint64_t, true>(pl, c, st) : launch_symbolic_sort_d<N, uint64_t, false>(pl, c, st);
+    return pl->diag ? launch_symbolic_sort_d<N, uint32_t, true>(pl, c, st) : launch_symbolic_sort_d<N, uint32_t, false>(pl, c, st);
+}
+
+template <typename V, int N, bool DIAG>
+spsyrk_status_t launch_numeric_map_d(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    if (count <= 0) return SPSYRK_OK;
+    constexpr int G = warp_class_group(N);
+    constexpr int NW = numeric_map_warps(N);
+    constexpr int ROWS = NW * (32 / G);
+    constexpr size_t smem = (size_t)ROWS * NumericMapSmem<V, N>::GROUP;
+    auto kern = numeric_map_warp_kernel<V, N, G, DIAG>;
+    SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const int64_t want = (count + ROWS - 1) / ROWS;
+    const int64_t cap = (int64_t)pl->sm_count * per_sm;
+    kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], pl->itemoff + pl->class_start[c],
+                                                               count, pl->map, c_rowptr, c_colidx, static_cast<V*>(c_vals));
+    note_launches(1);
+    return SPSYRK_OK;
+}
+
+template <typename V, int N>
+spsyrk_status_t launch_numeric_map(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    return pl->diag ? launch_numeric_map_d<V, N, true>(pl, c, c_rowptr, c_colidx, c_vals, st)
+                    : launch_numeric_map_d<V, N, false>(pl, c, c_rowptr, c_colidx, c_vals, st);
 }
 
 inline void mark(spsyrk_plan_s* pl, cudaEvent_t* ev, int i, cudaStream_t st) {
     if (pl->timing) cudaEventRecord(ev[i], st);
+}
+
+template <typename V>
+void launch_numeric_map_all(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    mark(pl, pl->ev_num, 1, st);
+    launch_numeric_map<V, 32>(pl, 1, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 2, st);
+    launch_numeric_map<V, 64>(pl, 2, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 3, st);
+    launch_numeric_map<V, 128>(pl, 3, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 4, st);
+    launch_numeric_map<V, 256>(pl, 4, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 5, st);
+    launch_numeric_map<V, 512>(pl, 5, c_rowptr, c_colidx, c_vals, st);
+    mark(pl, pl->ev_num, 6, st);
 }
 
 template <typename V, typename Key>
@@ -383,7 +494,8 @@ spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_
 
 template <typename V>
 spsyrk_status_t numeric_typed(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
-    if (pl->key64) launch_numeric_warp_all<V, uint64_t>(pl, c_rowptr, c_colidx, c_vals, st);
+    if (pl->map_filled) launch_numeric_map_all<V>(pl, c_rowptr, c_colidx, c_vals, st);
+    else if (pl->key64) launch_numeric_warp_all<V, uint64_t>(pl, c_rowptr, c_colidx, c_vals, st);
     else launch_numeric_warp_all<V, uint32_t>(pl, c_rowptr, c_colidx, c_vals, st);
     spsyrk_status_t s = launch_numeric_cta<V, 256>(pl, 6, BLOCK_ACC_SLOTS, c_rowptr, c_colidx, c_vals, st);
     if (s != SPSYRK_OK) return s;
@@ -449,7 +561,7 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     if (s != SPSYRK_OK) return fail(s);
     // 2. transpose: column histogram and scan give colptr; explicit row ids; stable radix sort by column
     if (nnz > 0) {
-        const unsigned hb = (unsigned)std::min<int64_t>((nnz + 255) / 256, 148 * 32);
+        const unsigned hb = (unsigned)std::min<int64_t>((nnz + 255) / 256, (int64_t)pl->sm_count * 32);
         column_histogram_kernel<<<hb, 256, 0, st>>>(d_colidx, nnz, P.n, pl->colcnt, P.err);
         note_launches(1);
     }
@@ -511,16 +623,18 @@ spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t* d_c_rowptr, int64_t
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int64_t rows = pl->dev.r1 - pl->dev.r0;
     if (rows > 0) SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->cnt, 0, (size_t)rows * sizeof(int32_t), st));
+    const bool with_map = use_map(pl);
+    pl->map_filled = false;
     mark(pl, pl->ev_sym, 1, st);
-    launch_symbolic_warp<32>(pl, 1, st);
+    if (with_map) launch_symbolic_sort<32>(pl, 1, st); else launch_symbolic_warp<32>(pl, 1, st);
     mark(pl, pl->ev_sym, 2, st);
-    launch_symbolic_warp<64>(pl, 2, st);
+    if (with_map) launch_symbolic_sort<64>(pl, 2, st); else launch_symbolic_warp<64>(pl, 2, st);
     mark(pl, pl->ev_sym, 3, st);
-    launch_symbolic_warp<128>(pl, 3, st);
+    if (with_map) launch_symbolic_sort<128>(pl, 3, st); else launch_symbolic_warp<128>(pl, 3, st);
     mark(pl, pl->ev_sym, 4, st);
-    launch_symbolic_warp<256>(pl, 4, st);
+    if (with_map) launch_symbolic_sort<256>(pl, 4, st); else launch_symbolic_warp<256>(pl, 4, st);
     mark(pl, pl->ev_sym, 5, st);
-    launch_symbolic_warp<512>(pl, 5, st);
+    if (with_map) launch_symbolic_sort<512>(pl, 5, st); else launch_symbolic_warp<512>(pl, 5, st);
     mark(pl, pl->ev_sym, 6, st);
     spsyrk_status_t s = launch_symbolic_cta<256>(pl, 6, st);
     if (s != SPSYRK_OK) return s;
@@ -536,6 +650,7 @@ spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t* d_c_rowptr, int64_t
     if (s != SPSYRK_OK) return s;
     *nnz_out = nnz;
     pl->have_symbolic = true;
+    pl->map_filled = with_map;
     return SPSYRK_OK;
 }
 
@@ -551,6 +666,21 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t* d_c_rowptr, in
         case SPSYRK_F32: return numeric_typed<float>(pl, d_c_rowptr, d_c_colidx, d_c_vals, st);
         default: return numeric_typed<int32_t>(pl, d_c_rowptr, d_c_colidx, d_c_vals, st);
     }
+}
+
+spsyrk_status_t spsyrk_plan_map_bytes(spsyrk_plan_t plan, size_t* bytes) {
+    if (!plan || !bytes) return SPSYRK_ERR_INVALID_ARG;
+    *bytes = (size_t)plan->map_items * sizeof(uint16_t);
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_plan_lend_map(spsyrk_plan_t plan, void* d_map, size_t bytes) {
+    if (!plan || (d_map && reinterpret_cast<uintptr_t>(d_map) % ALIGN)) return SPSYRK_ERR_INVALID_ARG;
+    plan->map = static_cast<uint16_t*>(d_map);
+    plan->map_bytes = d_map ? bytes : 0;
+    plan->map_filled = false;
+    plan->have_symbolic = false;
+    return SPSYRK_OK;
 }
 
 spsyrk_status_t spsyrk_plan_stats(spsyrk_plan_t plan, int64_t* work_total, int64_t class_rows[8]) {

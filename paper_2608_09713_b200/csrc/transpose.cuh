@@ -29,10 +29,18 @@ struct PlanDev {
     int64_t* colptr;
     int32_t* at_row;
     void* at_val;
+    void* at_rec;  // the same entries as interleaved (row id, value) records: ColRec<V>[nnz]
     uint2* desc;
     int64_t* work;  // per row of the range
     uint32_t* err;
 };
+
+// One entry of a column list as a record: what the light-row numeric kernel gathers (one aligned
+// asynchronous copy per entry, whatever the list's offset).
+template <typename V> struct ColRec;
+template <> struct alignas(16) ColRec<double> { int32_t j; int32_t pad; double v; };
+template <> struct alignas(8) ColRec<float> { int32_t j; float v; };
+template <> struct alignas(8) ColRec<int32_t> { int32_t j; int32_t v; };
 
 static __global__ void validate_rowptr_kernel(const int64_t* __restrict__ rowptr, int64_t m, int64_t nnz, uint32_t* err) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -77,6 +85,8 @@ struct EmitTransposeFinal {
         const int64_t cs = P.colptr[k];
         P.at_row[s] = (int32_t)row;
         static_cast<VB*>(P.at_val)[s] = val;  // bit copy of the value that travelled with the element
+        if constexpr (sizeof(VB) == 8) static_cast<uint4*>(P.at_rec)[s] = make_uint4(row, 0u, (uint32_t)val, (uint32_t)(val >> 32));
+        else static_cast<uint2*>(P.at_rec)[s] = make_uint2(row, (uint32_t)val);
         P.desc[p] = make_uint2((uint32_t)cs, P.mode == SPSYRK_TRIL ? (uint32_t)(s - cs) + 1u : (uint32_t)(P.colptr[k + 1] - cs));
     }
 };
@@ -106,7 +116,9 @@ static __global__ void __launch_bounds__(256) block_desc_kernel(PlanDev P, const
 //   class 0: no work; 1..5: w <= 32, 64, 128, 256, 512 and at most 32 nonzeros (one warp, register sort)
 //   6: w <= block_max (one 256-thread CTA, bitmap accumulator); 7: larger (one 1024-thread CTA)
 template <int G>
-static __global__ void __launch_bounds__(256) row_work_kernel(PlanDev P, uint8_t* __restrict__ cls, int64_t block_max,
+//   diag: the light-row kernels leave the diagonal products out of their item lists (lower-triangle mode
+//   over the whole column range), so a light row is classed by w minus its number of nonzeros
+static __global__ void __launch_bounds__(256) row_work_kernel(PlanDev P, uint8_t* __restrict__ cls, int64_t block_max, bool diag,
                                                         unsigned long long* __restrict__ work_total) {
     const int gl = threadIdx.x & (G - 1);
     const int64_t rows = P.r1 - P.r0;
@@ -127,8 +139,9 @@ static __global__ void __launch_bounds__(256) row_work_kernel(PlanDev P, uint8_t
         if (gid < rows && gl == 0) {
             P.work[gid] = w;
             uint8_t c;
+            const int64_t wl = diag ? w - deg : w;  // items of a light row
             if (w == 0) c = 0;
-            else if (deg <= 32 && w <= 512) c = w <= 32 ? 1 : w <= 64 ? 2 : w <= 128 ? 3 : w <= 256 ? 4 : 5;
+            else if (deg <= 32 && wl <= 512) c = wl <= 32 ? 1 : wl <= 64 ? 2 : wl <= 128 ? 3 : wl <= 256 ? 4 : 5;
             else c = w <= block_max ? 6 : 7;
             cls[gid] = c;
             mine += (unsigned long long)w;

@@ -39,14 +39,18 @@ def check_values(gpu_vals, ref, dtype):
 
 
 def run_and_compare(B, a: W.CSR, mode, r0=0, r1=None, cols=None, plan=None):
+    """Both ways of computing the light rows (with the item map lent to the plan and without it)
+    against the oracle; returns the result of the run with the map."""
     r1 = a.m if r1 is None else r1
     d = dev(a)
-    c_rowptr, c_colidx, c_vals, plan = B.tril_syrk(a.m, a.n, *d, mode=mode, row_begin=r0, row_end=r1, plan=plan)
-    torch.cuda.synchronize()
     ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, mode, r0, r1, cols=cols)
-    assert np.array_equal(c_rowptr.cpu().numpy(), ref.rowptr)
-    assert np.array_equal(c_colidx.cpu().numpy(), ref.colidx)
-    check_values(c_vals.cpu().numpy(), ref, a.vals.dtype)
+    for item_map in (False, True):
+        c_rowptr, c_colidx, c_vals, plan = B.tril_syrk(a.m, a.n, *d, mode=mode, row_begin=r0, row_end=r1, plan=plan,
+                                                       item_map=item_map)
+        torch.cuda.synchronize()
+        assert np.array_equal(c_rowptr.cpu().numpy(), ref.rowptr), f"item_map={item_map}"
+        assert np.array_equal(c_colidx.cpu().numpy(), ref.colidx), f"item_map={item_map}"
+        check_values(c_vals.cpu().numpy(), ref, a.vals.dtype)
     work, classes = B.spsyrk_plan_stats(plan)
     assert work == int(ref.work.sum())
     assert sum(classes) == r1 - r0
@@ -603,22 +607,24 @@ def test_rows_at_every_class_boundary(B):
     rng = np.random.default_rng(3)
     vals = rng.standard_normal(m)
     a = W.CSR(m, 1, np.arange(m + 1, dtype=np.int64), np.zeros(m, dtype=np.int32), vals)
-    rp, ci, cv, plan = B.tril_syrk(a.m, a.n, *dev(a))
-    i = np.arange(m + 1, dtype=np.int64)
-    assert np.array_equal(rp.cpu().numpy(), i * (i + 1) // 2)
-    work, classes = B.spsyrk_plan_stats(plan)
-    assert work == m * (m + 1) // 2
-    assert classes == [0, 32, 32, 64, 128, 256, 8192 - 512, m - 8192]
-    rows = torch.repeat_interleave(torch.arange(m, device="cuda"), torch.arange(1, m + 1, device="cuda"))
-    cols = torch.arange(ci.numel(), device="cuda") - rp[:-1][rows]
-    assert torch.equal(ci.long(), cols)
-    v = torch.from_numpy(vals).cuda()
-    assert torch.equal(cv, v[rows] * v[cols])                 # one product per entry: no rounding to differ in
-    for r in (0, 31, 32, 63, 64, 127, 128, 255, 256, 511, 512, 8191, 8192, m - 1):
-        ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, r, r + 1)
-        lo, hi = int(rp[r]), int(rp[r + 1])
-        assert np.array_equal(ci[lo:hi].cpu().numpy(), ref.colidx)
-        assert np.array_equal(cv[lo:hi].cpu().numpy(), ref.vals)
+    for item_map in (False, True):
+        rp, ci, cv, plan = B.tril_syrk(a.m, a.n, *dev(a), item_map=item_map)
+        i = np.arange(m + 1, dtype=np.int64)
+        assert np.array_equal(rp.cpu().numpy(), i * (i + 1) // 2)
+        work, classes = B.spsyrk_plan_stats(plan)
+        assert work == m * (m + 1) // 2
+        # a light row is classed by its products without the diagonal one (row i has i of them here)
+        assert classes == [0, 33, 32, 64, 128, 256, 8192 - 513, m - 8192]
+        rows = torch.repeat_interleave(torch.arange(m, device="cuda"), torch.arange(1, m + 1, device="cuda"))
+        cols = torch.arange(ci.numel(), device="cuda") - rp[:-1][rows]
+        assert torch.equal(ci.long(), cols)
+        v = torch.from_numpy(vals).cuda()
+        assert torch.equal(cv, v[rows] * v[cols])             # one product per entry: no rounding to differ in
+        for r in (0, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257, 511, 512, 513, 8191, 8192, m - 1):
+            ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, r, r + 1)
+            lo, hi = int(rp[r]), int(rp[r + 1])
+            assert np.array_equal(ci[lo:hi].cpu().numpy(), ref.colidx)
+            assert np.array_equal(cv[lo:hi].cpu().numpy(), ref.vals)
 
 
 def test_rows_with_33_nonzeros_leave_the_warp_classes(B):
