@@ -157,8 +157,8 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t *d_c_rowptr,
 
 /*
  * spsyrk_mirror - materialise F = C_L + C_L^T - D, the full symmetric matrix, from a complete
- * (untiled or re-assembled) lower triangle (Section III-A: "materializes it by transposing";
- * Section V-F: C = C_L + C_L^T - D).  Row i of F is row i of C_L followed by (r, c_ri) for
+ * (untiled or re-assembled) lower triangle (Section III-A: the full matrix, when it is needed, is
+ * obtained from the stored half by a transpose; Section V-F: C = C_L + C_L^T - D).  Row i of F is row i of C_L followed by (r, c_ri) for
  * every later row r that stores column i, ascending in r; values are bit copies, so F is
  * exactly symmetric and tril(F) == C_L.
  *
@@ -266,9 +266,10 @@ spsyrk_status_t spsyrk_symv(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
                             const void *d_x, void *d_y, void *cuda_stream);
 
 /*
- * spsyrk_mirror_rowptr_noalloc - the size step of spsyrk_mirror (step 2: d_f_rowptr[m + 1] and
- * *nnz_full_out of F = C_L + C_L^T - D) for callers that can neither allocate device memory nor
- * pass a workspace.  (The paper has no counterpart: this entry point exists for deployment only.)
+ * spsyrk_mirror_rowptr_noalloc - the sizes of F = C_L + C_L^T - D, that is d_f_rowptr[m + 1] as
+ * step 3 of spsyrk_mirror writes it and *nnz_full_out as step 2 returns it, for callers that can
+ * neither allocate device memory nor pass a workspace.  (The paper has no counterpart: this entry
+ * point exists for deployment only.)
  *
  * Who needs it: code that runs where device allocation is off limits - for instance a plug-in
  * inside a host application that has reserved the whole GPU for its own memory pool, or a service
@@ -290,8 +291,8 @@ spsyrk_status_t spsyrk_symv(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
  *     entry point clears what it accumulates into at the start of each call.  Two calls whose GPU
  *     work overlaps in time (different streams or threads) race on it: serialise them.
  *   - Synchronises the stream once (the entry count and the error word travel back).
- * Results are identical to step 2 of spsyrk_mirror.
- * Errors: INVALID_ARG, OVERFLOW, BAD_CSR (an entry above the diagonal), CUDA.
+ * The row pointers equal the ones step 3 of spsyrk_mirror writes, the count the one step 2 returns.
+ * Errors: INVALID_ARG, OVERFLOW, BAD_CSR (an entry above the diagonal, a decreasing row pointer), CUDA.
  */
 #define SPSYRK_NOALLOC_MAX_ROWS 1048576
 spsyrk_status_t spsyrk_mirror_rowptr_noalloc(int64_t m, const int64_t *d_l_rowptr, const int32_t *d_l_colidx,

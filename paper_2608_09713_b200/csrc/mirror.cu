@@ -18,7 +18,7 @@
 #include <algorithm>
 #include <mutex>
 
-#include "radix.cuh"
+#include "mirror_rec.cuh"
 
 using namespace spsyrk;
 
@@ -29,8 +29,14 @@ constexpr size_t ALIGN = 256;
 constexpr int MIRROR_RADIX_BITS = 8;
 
 struct MirrorWs {
-    uint32_t* ucnt;    // m: strictly-lower entries per column (allocation-free size step only)
+    uint32_t* diagf;   // m: 1 where the row stores its diagonal entry
     uint32_t* rowtot;  // m
+    int64_t* dcount;   // m + 1: diagonal entries of the rows before (exclusive prefix sums of diagf)
+    int64_t* fbase;    // m: l_rowptr[j + 1] - dcount[j + 1]
+    // 8-byte values: two record buffers and two digit-byte buffers (nnz_l entries each)
+    MirrorRec *rec_a, *rec_b;
+    uint8_t *dig_a, *dig_b;
+    int32_t* tile_rows;  // 2 per tile
     unsigned long long* seg_start;  // m: first sorted position of column j's strictly lower entries
     unsigned long long* seg_end;    // m: one past the last
     int64_t* partials;
@@ -53,20 +59,35 @@ size_t carve(MirrorWs* w, void* ws, int64_t m, int64_t nnz_l, size_t sv) {
     };
     const int64_t items = std::max<int64_t>(m, 1);
     const int64_t ne = std::max<int64_t>(nnz_l, 1);
-    const int64_t hist_n = (int64_t)(1 << MIRROR_RADIX_BITS) * std::max<int64_t>(radix_tiles(nnz_l), 1);
+    const int64_t hist_n = (int64_t)(1 << MIRROR_RADIX_BITS) * std::max<int64_t>(std::max(radix_tiles(nnz_l), mirror_tiles(nnz_l)), 1);
     MirrorWs t;
-    t.ucnt = (uint32_t*)take(items * 4);
+    t.diagf = (uint32_t*)take(items * 4);
     t.rowtot = (uint32_t*)take(items * 4);
+    t.dcount = (int64_t*)take((items + 1) * 8);
+    t.fbase = (int64_t*)take(items * 8);
     t.seg_start = (unsigned long long*)take(items * 8);
     t.seg_end = (unsigned long long*)take(items * 8);
     t.partials = (int64_t*)take(scan_partials_count(std::max<int64_t>(items + 1, hist_n)) * 8);
     t.err = (uint32_t*)take(8);  // [0] error word, [1] number of diagonal entries
-    t.key_a = (uint32_t*)take(ne * 4);
-    t.row_a = (uint32_t*)take(ne * 4);
-    t.key_b = (uint32_t*)take(ne * 4);
-    t.row_b = (uint32_t*)take(ne * 4);
-    t.val_a = take(ne * sv);
-    t.val_b = take(ne * sv);
+    t.key_a = t.row_a = t.key_b = t.row_b = nullptr;
+    t.val_a = t.val_b = nullptr;
+    t.rec_a = t.rec_b = nullptr;
+    t.dig_a = t.dig_b = nullptr;
+    t.tile_rows = nullptr;
+    if (sv == 8) {
+        t.rec_a = (MirrorRec*)take(ne * sizeof(MirrorRec));
+        t.rec_b = (MirrorRec*)take(ne * sizeof(MirrorRec));
+        t.dig_a = (uint8_t*)take(ne);
+        t.dig_b = (uint8_t*)take(ne);
+        t.tile_rows = (int32_t*)take(2 * std::max<int64_t>(mirror_tiles(nnz_l), 1) * 4);
+    } else {
+        t.key_a = (uint32_t*)take(ne * 4);
+        t.row_a = (uint32_t*)take(ne * 4);
+        t.key_b = (uint32_t*)take(ne * 4);
+        t.row_b = (uint32_t*)take(ne * 4);
+        t.val_a = take(ne * sv);
+        t.val_b = take(ne * sv);
+    }
     t.hist = (uint32_t*)take(hist_n * 4);
     t.offsets = (int64_t*)take((hist_n + 1) * 8);
     if (w) *w = t;
@@ -80,6 +101,7 @@ __global__ void __launch_bounds__(256) mirror_count_kernel(const int64_t* __rest
     const int gl = threadIdx.x & (G - 1);
     if (r >= m) return;
     const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
+    if (p1 < p0 && gl == 0) atomicOr(err, ERRW_BAD_ROWPTR);  // the row total below would wrap
     constexpr int UNR = 4;
     for (int64_t p = p0 + gl; p < p1; p += UNR * G) {
         int64_t j[UNR];
@@ -281,6 +303,110 @@ spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const i
     return SPSYRK_OK;
 }
 
+// 1 where row r stores its diagonal entry (rows are ascending: it is the last entry)
+__global__ void mirror_diag_flag_kernel(const int64_t* __restrict__ l_rowptr, const int32_t* __restrict__ l_colidx, int64_t m,
+                                        uint32_t* __restrict__ diagf) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= m) return;
+    const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
+    diagf[r] = (p1 > p0 && (int64_t)l_colidx[p1 - 1] == r) ? 1u : 0u;
+}
+
+__global__ void mirror_fbase_kernel(const int64_t* __restrict__ l_rowptr, const int64_t* __restrict__ dcount, int64_t m,
+                                    int64_t* __restrict__ fbase) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < m) fbase[j] = l_rowptr[j + 1] - dcount[j + 1];
+}
+
+// row lengths of F when the sorted segments include the diagonal entries
+__global__ void mirror_rowlen_diag_kernel(const int64_t* __restrict__ l_rowptr, const unsigned long long* __restrict__ seg_start,
+                                          const unsigned long long* __restrict__ seg_end, const uint32_t* __restrict__ diagf, int64_t m,
+                                          uint32_t* __restrict__ rowtot) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= m) return;
+    const unsigned long long s = seg_start[r], e = seg_end[r];
+    const uint32_t seg = e > s ? (uint32_t)(e - s) : 0u;
+    rowtot[r] = (uint32_t)(l_rowptr[r + 1] - l_rowptr[r]) + (seg >= diagf[r] ? seg - diagf[r] : 0u);
+}
+
+template <bool FROM_CSR, bool FINAL>
+cudaError_t launch_mirror_pass(const MirrorPassArgs& a, int64_t n, int shift, const int64_t* offsets, int64_t nt, cudaStream_t st) {
+    constexpr int BITS = MIRROR_RADIX_BITS;
+    auto kern = mirror_pass_kernel<BITS, FROM_CSR, FINAL>;
+    const size_t smem = MirrorPassSmem<BITS>::bytes();
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<(unsigned)nt, MR_THREADS, smem, st>>>(a, n, shift, offsets, nt);
+    note_launches(1);
+    return cudaGetLastError();
+}
+
+// 8-byte values: records, the first pass straight from C_L
+spsyrk_status_t mirror_fill_rec(const MirrorWs& w, int64_t m, int64_t nnz_l, const int64_t* l_rowptr, const int32_t* l_colidx,
+                                const void* l_vals, int64_t* f_rowptr, int32_t* f_colidx, void* f_vals, cudaStream_t st) {
+    constexpr int BITS = MIRROR_RADIX_BITS;
+    constexpr int NB = 1 << BITS;
+    const uint64_t* lv = static_cast<const uint64_t*>(l_vals);
+    uint64_t* fv = static_cast<uint64_t*>(f_vals);
+    const int g = group_width(nnz_l, m);
+    if (m > 0) {
+        SPSYRK_CUDA_TRY(cudaMemsetAsync(w.seg_start, 0xff, (size_t)m * 8, st));
+        SPSYRK_CUDA_TRY(cudaMemsetAsync(w.seg_end, 0, (size_t)m * 8, st));
+        mirror_diag_flag_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(l_rowptr, l_colidx, m, w.diagf);
+        note_launches(1);
+    }
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(w.diagf, m, w.dcount, w.partials, st));
+    if (m > 0 && nnz_l > 0) {
+        mirror_fbase_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(l_rowptr, w.dcount, m, w.fbase);
+        note_launches(1);
+        const int npass = (bits_for((uint64_t)(m - 1 > 0 ? m - 1 : 1)) + BITS - 1) / BITS;  // keys are column ids below m
+        const int64_t nt = mirror_tiles(nnz_l);
+        mirror_tile_rows_kernel<<<(unsigned)((2 * nt + 255) / 256), 256, 0, st>>>(l_rowptr, m, nnz_l, nt, w.tile_rows);
+        note_launches(1);
+        MirrorPassArgs a{};
+        a.l_rowptr = l_rowptr; a.l_colidx = l_colidx; a.l_vals = lv; a.m = m; a.tile_rows = w.tile_rows;
+        a.fbase = w.fbase; a.f_colidx = f_colidx; a.f_vals = fv; a.seg_start = w.seg_start; a.seg_end = w.seg_end;
+        a.dtotal = w.dcount + m; a.err = w.err;
+        for (int p = 0; p < npass; ++p) {
+            const bool first = p == 0, last = p == npass - 1;
+            const bool to_a = (p % 2) == 0;
+            const unsigned hb = (unsigned)((nt + MR_HIST_TILES - 1) / MR_HIST_TILES);
+            if (first) mirror_hist_key_kernel<BITS><<<hb, MR_THREADS, 0, st>>>(reinterpret_cast<const uint32_t*>(l_colidx), nnz_l, 0, w.hist, nt);
+            else radix_hist_u8_kernel<BITS><<<hb, MR_THREADS, 0, st>>>(to_a ? w.dig_b : w.dig_a, nnz_l, w.hist, nt);
+            note_launches(1);
+            SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(w.hist, (int64_t)NB * nt, w.offsets, w.partials, st));
+            a.src = to_a ? w.rec_b : w.rec_a;
+            a.dst = to_a ? w.rec_a : w.rec_b;
+            a.next_digit = to_a ? w.dig_a : w.dig_b;
+            cudaError_t e;
+            if (first && last) e = launch_mirror_pass<true, true>(a, nnz_l, p * BITS, w.offsets, nt, st);
+            else if (first) e = launch_mirror_pass<true, false>(a, nnz_l, p * BITS, w.offsets, nt, st);
+            else if (last) e = launch_mirror_pass<false, true>(a, nnz_l, p * BITS, w.offsets, nt, st);
+            else e = launch_mirror_pass<false, false>(a, nnz_l, p * BITS, w.offsets, nt, st);
+            SPSYRK_CUDA_TRY(e);
+        }
+    }
+    if (m > 0) {
+        mirror_rowlen_diag_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(l_rowptr, w.seg_start, w.seg_end, w.diagf, m, w.rowtot);
+        note_launches(1);
+    }
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(w.rowtot, m, f_rowptr, w.partials, st));
+    if (m > 0 && nnz_l > 0) {
+#define COPY(G) \
+    mirror_copy_lower_kernel<uint64_t, G><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(l_rowptr, l_colidx, lv, m, f_rowptr, f_colidx, fv)
+        switch (g) {
+            case 4: COPY(4); break;
+            case 8: COPY(8); break;
+            case 16: COPY(16); break;
+            default: COPY(32); break;
+        }
+#undef COPY
+        note_launches(1);
+    }
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    return SPSYRK_OK;
+}
+
 }  // namespace
 
 extern "C" spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype, const int64_t* d_l_rowptr,
@@ -320,14 +446,15 @@ extern "C" spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_
     // step 3: fill
     if (!d_f_vals || (nnz_l > 0 && !d_l_vals)) return SPSYRK_ERR_INVALID_ARG;
     switch (dtype) {
-        case SPSYRK_F64: return mirror_fill<uint64_t>(w, m, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_f_rowptr, d_f_colidx, d_f_vals, st);
+        case SPSYRK_F64: return mirror_fill_rec(w, m, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_f_rowptr, d_f_colidx, d_f_vals, st);
         default: return mirror_fill<uint32_t>(w, m, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_f_rowptr, d_f_colidx, d_f_vals, st);
     }
 }
 
 
 // ------------------------------------------------------------------------------------------
-// Allocation-free variant of the size step of spsyrk_mirror.
+// Allocation-free computation of F's row pointers and entry count (what steps 2 and 3 of
+// spsyrk_mirror deliver between them).
 //
 // Some callers have no device memory to lend and may not create any: a plug-in running inside a
 // host application that has claimed the whole GPU for its own memory pool, or a service loop that
@@ -400,7 +527,7 @@ extern "C" spsyrk_status_t spsyrk_mirror_rowptr_noalloc(int64_t m, const int64_t
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(&nnz, d_f_rowptr + m, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(&e, err, 4, cudaMemcpyDeviceToHost, st));
     SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
-    if (e & ERRW_UPPER) return SPSYRK_ERR_BAD_CSR;
+    if (e & (ERRW_UPPER | ERRW_BAD_ROWPTR)) return SPSYRK_ERR_BAD_CSR;
     *nnz_full_out = nnz;
     return SPSYRK_OK;
 }
