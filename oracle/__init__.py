@@ -52,6 +52,8 @@ def _load():
         lib.oracle_permute.argtypes = [i64, i64, p, p, p, p, p, p, p, p]
         lib.oracle_partition.argtypes = [i64, p, i64, p]
         lib.oracle_symv.restype = ctypes.c_int
+        lib.oracle_symm.argtypes = [i64, i64, p, p, p, p, p, p]
+        lib.oracle_symm.restype = ctypes.c_int
         for f in (lib.oracle_transpose, lib.oracle_syrk_rows, lib.oracle_mirror, lib.oracle_jaccard):
             f.restype = ctypes.c_int
         _lib = lib
@@ -175,6 +177,21 @@ def symv(m, l_rowptr, l_colidx, l_vals, x):
     rc = lib.oracle_symv(m, _ptr(l_rowptr), _ptr(l_colidx), _ptr(l_vals), _ptr(x), _ptr(y), _ptr(ay))
     assert rc == 0
     return y[:m], ay[:m]
+
+
+def symm(m, l_rowptr, l_colidx, l_vals, x):
+    """(Y, abs_Y): Y = C X = C_L X + (X^T C_L)^T - D X for a dense X of shape (m, p) from the lower
+    triangle (Section V-F, second equation); abs_Y holds the sums of the absolute contributions."""
+    lib = _load()
+    l_rowptr, l_colidx, l_vals = _c(l_rowptr, np.int64), _c(l_colidx, np.int32), _c(l_vals, np.float64)
+    x = _c(x, np.float64)
+    assert x.ndim == 2 and x.shape[0] == m
+    p = x.shape[1]
+    y = np.empty((max(m, 1), max(p, 1)), dtype=np.float64)
+    ay = np.empty_like(y)
+    rc = lib.oracle_symm(m, p, _ptr(l_rowptr), _ptr(l_colidx), _ptr(l_vals), _ptr(x), _ptr(y), _ptr(ay))
+    assert rc == 0
+    return y[:m, :p].copy(), ay[:m, :p].copy()
 
 
 def column_panel(m, rowptr, colidx, vals, k0, k1):

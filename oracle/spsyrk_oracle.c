@@ -210,6 +210,41 @@ int oracle_symv(int64_t m, const int64_t *l_rowptr, const int32_t *l_colidx, con
     return 0;
 }
 
+/* Y = C X for a dense row-major X (m x p) from the stored lower triangle (Section V-F, second
+ * equation): C X = C_L X + (X^T C_L)^T - D X.  Written as the three terms of the equation, each a
+ * plain loop over the stored entries; abs_y receives the sum of |c_rj| |x_jq| over all
+ * contributions of an output element, the scale for rounding comparisons.  Y and abs_y are
+ * row-major m x p. */
+int oracle_symm(int64_t m, int64_t p, const int64_t *l_rowptr, const int32_t *l_colidx, const double *l_vals,
+                const double *x, double *y, double *abs_y)
+{
+    for (int64_t e = 0; e < m * p; ++e) { y[e] = 0.0; abs_y[e] = 0.0; }
+    for (int64_t r = 0; r < m; ++r)                      /* C_L X: row r of Y += c_rj * row j of X */
+        for (int64_t q = l_rowptr[r]; q < l_rowptr[r + 1]; ++q) {
+            const int64_t j = l_colidx[q];
+            for (int64_t c = 0; c < p; ++c) {
+                y[r * p + c] += l_vals[q] * x[j * p + c];
+                abs_y[r * p + c] += fabs(l_vals[q] * x[j * p + c]);
+            }
+        }
+    for (int64_t r = 0; r < m; ++r)                      /* (X^T C_L)^T: row j of Y += c_rj * row r of X */
+        for (int64_t q = l_rowptr[r]; q < l_rowptr[r + 1]; ++q) {
+            const int64_t j = l_colidx[q];
+            for (int64_t c = 0; c < p; ++c) {
+                y[j * p + c] += l_vals[q] * x[r * p + c];
+                abs_y[j * p + c] += fabs(l_vals[q] * x[r * p + c]);
+            }
+        }
+    for (int64_t r = 0; r < m; ++r)                      /* - D X */
+        for (int64_t q = l_rowptr[r]; q < l_rowptr[r + 1]; ++q)
+            if (l_colidx[q] == r)
+                for (int64_t c = 0; c < p; ++c) {
+                    y[r * p + c] -= l_vals[q] * x[r * p + c];
+                    abs_y[r * p + c] += fabs(l_vals[q] * x[r * p + c]);
+                }
+    return 0;
+}
+
 /* Column panel A_s = A(:, [k0, k1)) as CSR with the column ids unchanged (Section III-A: the
  * diagonal block of C is a sum over s of SYRK(A_is), one term per column panel).  Rows keep
  * their order.  First call with out_colidx == NULL fills out_rowptr[m+1]; second call fills

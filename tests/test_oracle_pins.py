@@ -400,6 +400,46 @@ def test_symv_tiny_by_hand():
     assert list(y) == [47.0, 18.0, 140.0]
 
 
+@pytest.mark.parametrize("p", [1, 3, 8])
+def test_symm_equals_a_at_x(small_case, p):
+    """Section V-F, second equation: C X from the lower triangle equals A (A^T X) (the paper's own
+    alternative evaluation) and scipy's product of the mirrored matrix with X; one column is the
+    vector form."""
+    _, a, _, tril = small_case
+    rng = np.random.default_rng(80 + p)
+    x = rng.standard_normal((a.m, p))
+    y, ay = oracle.symm(a.m, tril.rowptr, tril.colidx, tril.vals, x)
+    A = sp.csr_matrix((a.vals.astype(np.float64), a.colidx, a.rowptr), shape=(a.m, a.n))
+    ref = A @ (A.T @ x)
+    absA = abs(A)
+    bound = absA @ (absA.T @ np.abs(x)) + 1e-300
+    assert np.all(np.abs(y - ref) <= 1e-12 * bound)
+    f_rowptr, f_colidx, f_vals = oracle.mirror(a.m, tril.rowptr, tril.colidx, tril.vals)
+    F = sp.csr_matrix((f_vals, f_colidx, f_rowptr), shape=(a.m, a.m))
+    assert np.all(np.abs(y - F @ x) <= 1e-13 * (ay + 1e-300))
+    for c in range(p):                                   # every column on its own is the vector identity
+        yc, _ = oracle.symv(a.m, tril.rowptr, tril.colidx, tril.vals, x[:, c])
+        assert np.array_equal(yc, y[:, c])
+
+
+def test_symm_tiny_by_hand():
+    # C_L = [[5], [., 9], [14, ., 42]], so C = [[5, 0, 14], [0, 9, 0], [14, 0, 42]];
+    # X = [[1, 0], [2, 1], [3, -1]]: C X = [[5 + 42, -14], [18, 9], [14 + 126, -42]]
+    y, ay = oracle.symm(3, [0, 1, 2, 4], [0, 1, 0, 2], [5.0, 9.0, 14.0, 42.0], [[1.0, 0.0], [2.0, 1.0], [3.0, -1.0]])
+    assert y.tolist() == [[47.0, -14.0], [18.0, 9.0], [140.0, -42.0]]
+    # a wrong sign on the diagonal term or a missing reflected term changes these; a transposed X cannot be passed
+    assert ay.tolist() == [[5.0 + 42.0 + 5.0 + 5.0, 14.0], [18.0 * 3, 9.0 * 3], [14.0 + 126.0 + 126.0 + 126.0, 42.0 * 3]]
+
+
+def test_symm_degenerate_shapes():
+    y, _ = oracle.symm(0, [0], [], [], np.zeros((0, 4)))
+    assert y.shape == (0, 4)
+    y, _ = oracle.symm(2, [0, 0, 0], [], [], np.ones((2, 3)))       # an empty triangle gives zeros
+    assert np.array_equal(y, np.zeros((2, 3)))
+    y, _ = oracle.symm(2, [0, 1, 2], [0, 1], [2.0, 3.0], np.array([[1.0], [4.0]]))   # diagonal only: counted once
+    assert y.tolist() == [[2.0], [12.0]]
+
+
 # ------------------------------------------------- accumulating form over column panels
 def dense_add_reference(x, sx, y, sy):
     """Dense statement of Z = X + Y with explicit structure masks: stored iff stored in either."""
