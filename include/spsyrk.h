@@ -266,6 +266,21 @@ spsyrk_status_t spsyrk_symv(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,
                             const void *d_x, void *d_y, void *cuda_stream);
 
 /*
+ * spsyrk_symm - Y = C X for a dense X from the stored lower triangle alone,
+ *     C X = C_L X + (X^T C_L)^T - D X        (Section V-F, second equation: the matrix form of the
+ * triangular product; unlike the vector form it cannot be replaced by A (A^T X) without possibly
+ * more arithmetic than (A A^T) X, so consuming C_L directly is the form worth having).
+ * C_L is any lower-triangular CSR (diagonal included) of F64 or F32 values with m rows; d_x and d_y are
+ * dense row-major device matrices of the same type, m rows by p columns (element (i, c) at i * p + c);
+ * Y is overwritten and must not alias X.  The reflected contributions are accumulated with atomic
+ * adds, so the last bits of Y can differ from run to run.  Columns are processed eight at a time
+ * (C_L is read once per eight columns of X).  Asynchronous.  Errors: INVALID_ARG, CUDA.
+ */
+spsyrk_status_t spsyrk_symm(int64_t m, int64_t p, int64_t nnz_l, spsyrk_dtype_t dtype,
+                            const int64_t *d_l_rowptr, const int32_t *d_l_colidx, const void *d_l_vals,
+                            const void *d_x, void *d_y, void *cuda_stream);
+
+/*
  * spsyrk_mirror_rowptr_noalloc - the sizes of F = C_L + C_L^T - D, that is d_f_rowptr[m + 1] as
  * step 3 of spsyrk_mirror writes it and *nnz_full_out as step 2 returns it, for callers that can
  * neither allocate device memory nor pass a workspace.  (The paper has no counterpart: this entry

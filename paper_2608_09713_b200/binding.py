@@ -54,6 +54,8 @@ _lib.spsyrk_mirror_rowptr_noalloc.argtypes = [_i64, _vp, _vp, _vp, _i64p, _vp]
 _lib.spsyrk_mirror_rowptr_noalloc.restype = _int
 _lib.spsyrk_symv.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_symv.restype = _int
+_lib.spsyrk_symm.argtypes = [_i64, _i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.spsyrk_symm.restype = _int
 _lib.spsyrk_jaccard.argtypes = [_i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_plan_stats.argtypes = [_vp, _i64p, _i64p]
 _lib.spsyrk_plan_buffers.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]
@@ -368,6 +370,18 @@ def spsyrk_symv(m, l_rowptr, l_colidx, l_vals, x, y=None, stream=None):
         y = torch.empty(m, dtype=x.dtype, device=x.device)
     _check(_lib.spsyrk_symv(m, l_colidx.numel(), _DTYPE_CODE[l_vals.dtype], _p(l_rowptr), _p(l_colidx), _p(l_vals),
                             _p(x), _p(y), _stream(stream)), "spsyrk_symv")
+    return y
+
+
+def spsyrk_symm(m, l_rowptr, l_colidx, l_vals, x, y=None, stream=None):
+    """Y = C X = C_L X + (X^T C_L)^T - D X for a dense row-major X of shape (m, p), from the lower triangle only."""
+    _dev_check(l_rowptr, l_colidx, l_vals, x, y)
+    assert x.dtype == l_vals.dtype and x.dim() == 2 and x.shape[0] == m
+    p = x.shape[1]
+    if y is None:
+        y = torch.empty((m, p), dtype=x.dtype, device=x.device)
+    _check(_lib.spsyrk_symm(m, p, l_colidx.numel(), _DTYPE_CODE[l_vals.dtype], _p(l_rowptr), _p(l_colidx), _p(l_vals),
+                            _p(x), _p(y), _stream(stream)), "spsyrk_symm")
     return y
 
 

@@ -57,6 +57,90 @@ spsyrk_status_t symv_typed(int64_t m, int64_t nnz_l, const int64_t* l_rowptr, co
 
 }  // namespace
 
+namespace {
+
+// Y = C_L X + (X^T C_L)^T - D X for a dense row-major X (m x p), columns in chunks of PC: G lanes share a
+// row of C_L; for every stored entry (r, j, v) a lane adds v * X[j, c0..c0+PC) to its partial row of Y
+// (registers) and, when j != r, v * X[r, c0..c0+PC) to row j of Y (atomic adds): the diagonal is counted
+// once and C_L^T is never formed.  The rows of X are read as contiguous pieces of PC values.
+template <typename V, int G, int PC>
+__global__ void __launch_bounds__(256) symm_kernel(int64_t m, int64_t p, int64_t c0, const int64_t* __restrict__ l_rowptr,
+                                                   const int32_t* __restrict__ l_colidx, const V* __restrict__ l_vals,
+                                                   const V* __restrict__ x, V* __restrict__ y) {
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    const int gl = threadIdx.x & (G - 1);
+    const int pc = (int)min((int64_t)PC, p - c0);  // columns of this chunk
+    V acc[PC], xr[PC];
+#pragma unroll
+    for (int c = 0; c < PC; ++c) { acc[c] = V(0); xr[c] = V(0); }
+    if (r < m) {
+#pragma unroll
+        for (int c = 0; c < PC; ++c)
+            if (c < pc) xr[c] = x[r * p + c0 + c];
+        const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
+        for (int64_t q = p0 + gl; q < p1; q += G) {
+            const int64_t j = l_colidx[q];
+            const V v = l_vals[q];
+            const V* xj = x + j * p + c0;
+            V* yj = y + j * p + c0;
+#pragma unroll
+            for (int c = 0; c < PC; ++c) {
+                if (c < pc) {
+                    acc[c] += v * xj[c];
+                    if (j != r) atomicAdd(&yj[c], v * xr[c]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < PC; ++c) {
+#pragma unroll
+        for (int o = G / 2; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(FULL_MASK, acc[c], o);
+    }
+    if (r < m && gl == 0) {
+#pragma unroll
+        for (int c = 0; c < PC; ++c)
+            if (c < pc) atomicAdd(&y[r * p + c0 + c], acc[c]);
+    }
+}
+
+template <typename V>
+spsyrk_status_t symm_typed(int64_t m, int64_t p, int64_t nnz_l, const int64_t* l_rowptr, const int32_t* l_colidx, const void* l_vals,
+                           const void* x, void* y, cudaStream_t st) {
+    SPSYRK_CUDA_TRY(cudaMemsetAsync(y, 0, (size_t)m * (size_t)p * sizeof(V), st));
+    const V* lv = static_cast<const V*>(l_vals);
+    const V* xv = static_cast<const V*>(x);
+    V* yv = static_cast<V*>(y);
+    constexpr int PC = 8;
+    for (int64_t c0 = 0; c0 < p; c0 += PC) {
+#define SYMM(G) symm_kernel<V, G, PC><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(m, p, c0, l_rowptr, l_colidx, lv, xv, yv)
+        switch (group_width(nnz_l, m)) {
+            case 4: SYMM(4); break;
+            case 8: SYMM(8); break;
+            case 16: SYMM(16); break;
+            default: SYMM(32); break;
+        }
+#undef SYMM
+        note_launches(1);
+    }
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    return SPSYRK_OK;
+}
+
+}  // namespace
+
+extern "C" spsyrk_status_t spsyrk_symm(int64_t m, int64_t p, int64_t nnz_l, spsyrk_dtype_t dtype, const int64_t* d_l_rowptr,
+                                       const int32_t* d_l_colidx, const void* d_l_vals, const void* d_x, void* d_y,
+                                       void* cuda_stream) {
+    if (m < 0 || p < 0 || nnz_l < 0 || !d_l_rowptr || (m > 0 && p > 0 && (!d_x || !d_y)) || (nnz_l > 0 && (!d_l_colidx || !d_l_vals)))
+        return SPSYRK_ERR_INVALID_ARG;
+    if (dtype != SPSYRK_F64 && dtype != SPSYRK_F32) return SPSYRK_ERR_INVALID_ARG;
+    if (m == 0 || p == 0) return SPSYRK_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    return dtype == SPSYRK_F64 ? symm_typed<double>(m, p, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_x, d_y, st)
+                               : symm_typed<float>(m, p, nnz_l, d_l_rowptr, d_l_colidx, d_l_vals, d_x, d_y, st);
+}
+
 extern "C" spsyrk_status_t spsyrk_symv(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype, const int64_t* d_l_rowptr,
                                        const int32_t* d_l_colidx, const void* d_l_vals, const void* d_x, void* d_y,
                                        void* cuda_stream) {

@@ -419,6 +419,35 @@ def test_symv(B, idx):
     assert np.all(np.abs(y.astype(np.float64) - exp) <= tol * (scale + 1e-300))
 
 
+@pytest.mark.parametrize("idx", [1, 3, 4, 5])
+@pytest.mark.parametrize("p", [1, 8, 33])
+def test_symm(B, idx, p):
+    """Y = C_L X + (X^T C_L)^T - D X (Section V-F, second equation) against the oracle, element by element."""
+    a = W.small(idx)
+    (rp, ci, cv), ref, _ = run_and_compare(B, a, 0)
+    rng = np.random.default_rng(20 + p)
+    x = rng.standard_normal((a.m, p)).astype(a.vals.dtype)
+    y = B.spsyrk_symm(a.m, rp, ci, cv, torch.from_numpy(x).cuda()).cpu().numpy()
+    exp, scale = oracle.symm(a.m, rp.cpu().numpy(), ci.cpu().numpy(), cv.cpu().numpy().astype(np.float64), x.astype(np.float64))
+    tol = 1e-12 if a.vals.dtype == np.float64 else 2e-5
+    assert y.shape == exp.shape
+    assert np.all(np.abs(y.astype(np.float64) - exp) <= tol * (scale + 1e-300))
+    if p == 1:                                             # one column is the vector form
+        yv = B.spsyrk_symv(a.m, rp, ci, cv, torch.from_numpy(x[:, 0].copy()).cuda()).cpu().numpy()
+        assert np.all(np.abs(yv.astype(np.float64) - exp[:, 0]) <= tol * (scale[:, 0] + 1e-300))
+
+
+def test_symm_degenerate(B):
+    z = (torch.zeros(1, dtype=torch.int64, device="cuda"), torch.zeros(0, dtype=torch.int32, device="cuda"),
+         torch.zeros(0, dtype=torch.float64, device="cuda"))
+    assert B.spsyrk_symm(0, *z, torch.zeros((0, 3), dtype=torch.float64, device="cuda")).shape == (0, 3)
+    rp = torch.tensor([0, 1, 2], dtype=torch.int64, device="cuda")
+    ci = torch.tensor([0, 1], dtype=torch.int32, device="cuda")
+    cv = torch.tensor([2.0, 3.0], dtype=torch.float64, device="cuda")
+    x = torch.tensor([[1.0, -1.0], [4.0, 0.5]], dtype=torch.float64, device="cuda")
+    assert B.spsyrk_symm(2, rp, ci, cv, x).cpu().tolist() == [[2.0, -2.0], [12.0, 1.5]]    # the diagonal counts once
+
+
 # ------------------------------------------- accumulating form over column panels (Section III-A, Algorithm 2)
 def _np(*ts):
     return [t.cpu().numpy() for t in ts]
@@ -641,3 +670,75 @@ def test_rows_with_33_nonzeros_leave_the_warp_classes(B):
     _, classes = B.spsyrk_plan_stats(plan)
     assert sum(classes[6:]) >= m // 2
     run_and_compare(B, a, 1)
+
+
+# ------------------------------------------------ heavy rows beyond one bitmap chunk (more than 2^20 rows)
+def _hub_matrix(dtype):
+    """Three uniform columns per row, one column stored in 9000 scattered rows and three rows of 40
+    nonzeros near the end, with more than 2^20 rows: the heavy rows sit at high row indices, so their
+    output range spans several bitmap chunks of the one-CTA-per-row kernels in both passes."""
+    m = n = (1 << 20) + 1000
+    rng = np.random.default_rng(77)
+    cols = rng.integers(0, n, size=(m, 3))
+    hub_rows = np.sort(rng.choice(m, size=9000, replace=False))
+    wide_rows = np.array([m - 700, m - 350, m - 2])
+    lists = {}
+    for r in hub_rows:
+        lists[int(r)] = np.union1d(cols[r], [7])
+    for r in wide_rows:
+        base = lists.get(int(r), np.unique(cols[r]))
+        lists[int(r)] = np.union1d(base, rng.choice(n, size=40, replace=False))
+    rowptr = np.zeros(m + 1, dtype=np.int64)
+    srt = np.sort(cols, axis=1)
+    dup = (srt[:, 1:] == srt[:, :-1])
+    base_deg = 3 - dup.sum(axis=1)
+    degs = base_deg.copy()
+    for r, l in lists.items():
+        degs[r] = l.size
+    np.cumsum(degs, out=rowptr[1:])
+    colidx = np.empty(rowptr[-1], dtype=np.int32)
+    keep = np.ones((m, 3), dtype=bool)
+    keep[:, 1:] &= ~dup
+    plain = np.ones(m, dtype=bool)
+    plain[list(lists.keys())] = False
+    # rows without additions: their distinct sorted columns, written in one go
+    sel = keep & plain[:, None]
+    pos = (rowptr[:-1][:, None] + np.cumsum(keep, axis=1) - 1)
+    colidx[pos[sel]] = srt[sel]
+    for r, l in lists.items():
+        colidx[rowptr[r]:rowptr[r + 1]] = l
+    if np.issubdtype(dtype, np.integer):
+        vals = rng.integers(1, 4, size=colidx.size).astype(dtype)
+    else:
+        vals = rng.standard_normal(colidx.size).astype(dtype)
+    return W.CSR(m, n, rowptr, colidx, vals), hub_rows, wide_rows
+
+
+@pytest.mark.parametrize("dtype", [np.float64, np.int32])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_heavy_rows_beyond_one_chunk(B, dtype, mode):
+    a, hub_rows, wide_rows = _hub_matrix(dtype)
+    assert np.all(np.diff(a.rowptr) >= 1)
+    d = dev(a)
+    rp, ci, cv, plan = B.tril_syrk(a.m, a.n, *d, mode=mode)
+    _, classes = B.spsyrk_plan_stats(plan)
+    assert classes[6] > 0 and classes[7] > 0, classes      # both one-CTA-per-row classes are exercised
+    rp_h = rp.cpu().numpy()
+    cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
+    # rows of every kind: hub rows early (short prefix), in the middle of the block class (one and several
+    # accumulator tiles), in the large class, the rows with more than 32 nonzeros, and a few light neighbours
+    picks = [hub_rows[10], hub_rows[600], hub_rows[3000], hub_rows[5000], hub_rows[8000], hub_rows[8500], hub_rows[-1],
+             *wide_rows, hub_rows[-1] - 1 if hub_rows[-1] - 1 not in hub_rows else hub_rows[-1] + 1, a.m - 1]
+    for r in picks:
+        r = int(r)
+        ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, mode, r, r + 1, cols=cols)
+        lo, hi = int(rp_h[r]), int(rp_h[r + 1])
+        assert hi - lo == ref.nnz, (r, hi - lo, ref.nnz)
+        assert np.array_equal(ci[lo:hi].cpu().numpy(), ref.colidx), r
+        check_values(cv[lo:hi].cpu().numpy(), ref, a.vals.dtype)
+    # every row's count against the closed form where there is one: a hub row's lower part holds the hub
+    # rows before it (through column 7), itself, and what its other columns add
+    if mode == 0:
+        cnt = np.diff(rp_h)
+        rank = np.arange(1, hub_rows.size + 1)
+        assert np.all(cnt[hub_rows] >= rank)
