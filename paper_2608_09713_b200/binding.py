@@ -13,7 +13,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libspsyrk.so")
+# SPSYRK_LIBRARY selects another build of the same library (the bounds-checked one, libspsyrk_checked.so)
+LIB_PATH = os.environ.get("SPSYRK_LIBRARY") or os.path.join(_HERE, "libspsyrk.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

@@ -9,6 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspsyrk.so")
+LIB_CHECKED = os.path.join(HERE, "libspsyrk_checked.so")  # same sources with -DSPSYRK_CHECKED (bounds-checked indices)
 SOURCES = ["api.cu", "mirror.cu", "jaccard.cu", "symv.cu", "accumulate.cu", "permute.cu", "host.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",
@@ -21,13 +22,17 @@ def _newest_source_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build_cuda(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
-        return LIB
+def build_cuda(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compile the library; `checked` builds the bounds-checked variant (libspsyrk_checked.so) instead."""
+    lib = LIB_CHECKED if checked else LIB
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _newest_source_mtime():
+        return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    objdir = os.path.join(HERE, "build")
+    objdir = os.path.join(HERE, "build", "checked" if checked else "release")
     os.makedirs(objdir, exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
+    if checked:
+        extra.append("-DSPSYRK_CHECKED")
 
     def compile_one(src):
         obj = os.path.join(objdir, src.replace(".cu", ".o"))
@@ -36,9 +41,9 @@ def build_cuda(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
         objs = list(ex.map(compile_one, SOURCES))
-    subprocess.check_call([nvcc, "-shared", "-o", LIB, *objs, "-lcudart"])
-    return LIB
+    subprocess.check_call([nvcc, "-shared", "-o", lib, *objs, "-lcudart"])
+    return lib
 
 
 if __name__ == "__main__":
-    print(build_cuda(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_cuda(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

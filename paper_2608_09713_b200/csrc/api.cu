@@ -214,11 +214,11 @@ spsyrk_status_t sort_by_column(spsyrk_plan_s* pl, cudaStream_t st) {
         if (p == npass - 1) {
             EmitTransposeFinal<VB> emit{P};
             SPSYRK_CUDA_TRY((radix_pass3<BITS, VB>(src_key, src_row, src_val, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
-                                                   pl->partials, emit, st)));
+                                                   pl->partials, emit, P.err, st)));
         } else {
             EmitArrays3<VB> emit{dst_key, dst_row, dst_val, dst_pos};
             SPSYRK_CUDA_TRY((radix_pass3<BITS, VB>(src_key, src_row, src_val, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
-                                                   pl->partials, emit, st)));
+                                                   pl->partials, emit, P.err, st)));
         }
         src_key = dst_key;
         src_row = dst_row;
@@ -504,7 +504,11 @@ spsyrk_status_t numeric_typed(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_
     if (s != SPSYRK_OK) return s;
     mark(pl, pl->ev_num, 8, st);
     SPSYRK_CUDA_TRY(cudaGetLastError());
+#ifdef SPSYRK_CHECKED
+    return read_err(pl, st);  // the bounds-checked build reports a skipped access at once (synchronises)
+#else
     return SPSYRK_OK;
+#endif
 }
 
 }  // namespace

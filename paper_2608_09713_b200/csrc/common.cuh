@@ -20,6 +20,16 @@ enum : uint32_t {
     ERRW_UPPER = 16u,
 };
 
+// Bounds-checked build (-DSPSYRK_CHECKED, a second library next to the regular one): every index into a
+// shared-memory accumulator, hash or landing slot and every output offset that the kernels compute is
+// tested first; a violation sets ERRW_INTERNAL in the device error word and the access is skipped, so the
+// caller gets SPSYRK_ERR_INTERNAL instead of a memory fault.  In the regular build the test is `true`.
+#ifdef SPSYRK_CHECKED
+#define SPSYRK_IN_RANGE(cond, errptr) ((cond) ? true : (atomicOr((errptr), ::spsyrk::ERRW_INTERNAL), false))
+#else
+#define SPSYRK_IN_RANGE(cond, errptr) true
+#endif
+
 constexpr int NCLASS = 8;  // row / column classes produced by the binning pass
 
 // kernel-launch bookkeeping behind spsyrk_launch_count (defined in api.cu)

@@ -271,10 +271,10 @@ spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const i
             V* dst_val = static_cast<V*>(to_a ? w.val_a : w.val_b);
             if (p == npass - 1) {
                 EmitMirrorFinal<V> emit{l_rowptr, f_colidx, fv, w.seg_start, w.seg_end, (uint32_t)m};
-                SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+                SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, w.err, st)));
             } else {
                 EmitArrays<V> emit{dst_key, dst_row, dst_val};
-                SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+                SPSYRK_CUDA_TRY((radix_pass<BITS, V>(src_key, src_row, src_val, nnz_l, p * BITS, w.hist, w.offsets, w.partials, emit, w.err, st)));
             }
             src_key = dst_key;
             src_row = dst_row;
@@ -300,6 +300,14 @@ spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const i
         note_launches(1);
     }
     SPSYRK_CUDA_TRY(cudaGetLastError());
+#ifdef SPSYRK_CHECKED
+    {
+        uint32_t e = 0;  // the bounds-checked build reports a skipped access at once (synchronises)
+        SPSYRK_CUDA_TRY(cudaMemcpyAsync(&e, w.err, 4, cudaMemcpyDeviceToHost, st));
+        SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
+        if (e & ERRW_INTERNAL) return SPSYRK_ERR_INTERNAL;
+    }
+#endif
     return SPSYRK_OK;
 }
 
@@ -404,6 +412,14 @@ spsyrk_status_t mirror_fill_rec(const MirrorWs& w, int64_t m, int64_t nnz_l, con
         note_launches(1);
     }
     SPSYRK_CUDA_TRY(cudaGetLastError());
+#ifdef SPSYRK_CHECKED
+    {
+        uint32_t e = 0;  // the bounds-checked build reports a skipped access at once (synchronises)
+        SPSYRK_CUDA_TRY(cudaMemcpyAsync(&e, w.err, 4, cudaMemcpyDeviceToHost, st));
+        SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
+        if (e & ERRW_INTERNAL) return SPSYRK_ERR_INTERNAL;
+    }
+#endif
     return SPSYRK_OK;
 }
 

@@ -285,7 +285,8 @@ __global__ void __launch_bounds__(MR_THREADS, MR_MIN_CTAS) mirror_pass_kernel(Mi
         const int t = warp * MR_CHUNK + i * 32 + lane;
         if (t < tile_n) {
             const uint32_t q = mycount[rk[i] >> 16] + (rk[i] & 0xffffu);
-            reinterpret_cast<uint4*>(s_rec)[q] = make_uint4(k[i], a[i], (uint32_t)b[i], (uint32_t)(b[i] >> 32));
+            if (SPSYRK_IN_RANGE(q < (uint32_t)MR_TILE, A.err))
+                reinterpret_cast<uint4*>(s_rec)[q] = make_uint4(k[i], a[i], (uint32_t)b[i], (uint32_t)(b[i] >> 32));
         }
     }
     __syncthreads();
@@ -294,6 +295,7 @@ __global__ void __launch_bounds__(MR_THREADS, MR_MIN_CTAS) mirror_pass_kernel(Mi
         MirrorRec r;
         r.key = r4.x; r.row = r4.y; r.val = (uint64_t)r4.z | ((uint64_t)r4.w << 32);
         const int64_t dest = goff[(r.key >> shift) & (NB - 1)] + q;
+        if (!SPSYRK_IN_RANGE(dest >= 0 && dest < n, A.err)) continue;
         if (!FINAL) {
             reinterpret_cast<uint4*>(A.dst)[dest] = r4;
             A.next_digit[dest] = (uint8_t)((r.key >> (shift + BITS)) & (NB - 1));

@@ -67,13 +67,17 @@ __global__ void check_permutation_kernel(const int32_t* __restrict__ perm, int64
     else if (atomicExch(&seen[v], 1u) != 0u) atomicOr(err, ERRW_BAD_COL);
 }
 
-__global__ void permuted_lengths_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ rperm, int64_t m,
+// Also the row-pointer checks of the whole call: rowptr[0] = 0, rowptr[m] = nnz, non-decreasing, inside [0, nnz] -
+// the expand kernel indexes arrays of nnz entries with these positions.
+__global__ void permuted_lengths_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ rperm, int64_t m, int64_t nnz,
                                         uint32_t* __restrict__ len, uint32_t* err) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= m) return;
-    const int64_t l = rowptr[i + 1] - rowptr[i];
+    const int64_t a = rowptr[i], b = rowptr[i + 1];
+    const int64_t l = b - a;
     const int64_t r = rperm[i];
-    if (l < 0 || l > 0x7fffffffLL) atomicOr(err, ERRW_BAD_ROWPTR);
+    if (i == 0 && (rowptr[0] != 0 || rowptr[m] != nnz)) atomicOr(err, ERRW_BAD_ROWPTR);
+    if (l < 0 || a < 0 || b > nnz) atomicOr(err, ERRW_BAD_ROWPTR);
     else if (r >= 0 && r < m) len[r] = (uint32_t)l;
 }
 
@@ -131,7 +135,7 @@ spsyrk_status_t permute_sort(const PermuteWs& w, int64_t m, int64_t n, int64_t n
         const int npass = (bits_for((uint64_t)std::max<int64_t>(n - 1, 1)) + BITS - 1) / BITS;
         for (int p = 0; p < npass; ++p) {
             EmitArrays<V> emit{other_key(), other_pay(), other_val()};
-            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(key, pay, val, nnz, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(key, pay, val, nnz, p * BITS, w.hist, w.offsets, w.partials, emit, w.err, st)));
             key = emit.keys; pay = emit.pa; val = emit.pb;
             in_a = !in_a;
         }
@@ -142,13 +146,13 @@ spsyrk_status_t permute_sort(const PermuteWs& w, int64_t m, int64_t n, int64_t n
     for (int p = 0; p < npass; ++p) {
         if (p == npass - 1) {
             EmitPermuted<V> emit{b_colidx, static_cast<V*>(b_vals)};
-            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(key, pay, val, nnz, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(key, pay, val, nnz, p * BITS, w.hist, w.offsets, w.partials, emit, w.err, st)));
         } else {
             // the roles of the two uint32 buffers of a pair are swapped with the arrays
             uint32_t* dk = in_a ? w.pay_b : w.pay_a;
             uint32_t* dp = in_a ? w.key_b : w.key_a;
             EmitArrays<V> emit{dk, dp, other_val()};
-            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(key, pay, val, nnz, p * BITS, w.hist, w.offsets, w.partials, emit, st)));
+            SPSYRK_CUDA_TRY((radix_pass<BITS, V>(key, pay, val, nnz, p * BITS, w.hist, w.offsets, w.partials, emit, w.err, st)));
             key = dk; pay = dp; val = emit.pb;
             in_a = !in_a;
         }
@@ -192,7 +196,7 @@ extern "C" spsyrk_status_t spsyrk_permute(int64_t m, int64_t n, int64_t nnz, sps
     }
     if (m > 0) {
         SPSYRK_CUDA_TRY(cudaMemsetAsync(w.len, 0, (size_t)m * 4, st));
-        permuted_lengths_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(d_rowptr, d_rperm, m, w.len, w.err);
+        permuted_lengths_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(d_rowptr, d_rperm, m, nnz, w.len, w.err);
         note_launches(1);
     }
     SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(w.len, m, d_b_rowptr, w.partials, st));

@@ -71,6 +71,7 @@ struct RadixSmem {
     }
 };
 
+// `err` is the device error word of the caller (used by the bounds-checked build only).
 // Emit(dest, key, pa, pb) is called once per element with its position `dest` in the order sorted
 // by the digits seen so far.  pa == nullptr (pb == nullptr) means "this payload is the element's own
 // index".
@@ -85,7 +86,7 @@ template <int BITS, typename PB, typename Emit, bool HAS_PC = false>
 __global__ void __launch_bounds__(RX_THREADS, 2) radix_scatter_kernel(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pa,
                                                                       const PB* __restrict__ pb, const uint32_t* __restrict__ pc,
                                                                       int64_t n, int shift, const int64_t* __restrict__ goff_all,
-                                                                      int64_t ntiles, Emit emit) {
+                                                                      int64_t ntiles, Emit emit, uint32_t* err) {
     constexpr int NB = 1 << BITS;
     static_assert(BITS <= 12, "digit width");
     extern __shared__ __align__(16) unsigned char rx_smem[];
@@ -187,6 +188,7 @@ __global__ void __launch_bounds__(RX_THREADS, 2) radix_scatter_kernel(const uint
         const int t = warp * RX_CHUNK + i * 32 + lane;
         if (t < tile_n) {
             const uint32_t q = mycount[rk[i] >> 16] + (rk[i] & 0xffffu);
+            if (!SPSYRK_IN_RANGE(q < (uint32_t)RX_TILE, err)) continue;
             s_key[q] = k[i];
             s_pa[q] = a[i];
             s_pb[q] = b[i];
@@ -198,6 +200,7 @@ __global__ void __launch_bounds__(RX_THREADS, 2) radix_scatter_kernel(const uint
     for (int q = tid; q < tile_n; q += RX_THREADS) {
         const uint32_t key = s_key[q];
         const int64_t dest = goff[(key >> shift) & (NB - 1)] + q;
+        if (!SPSYRK_IN_RANGE(dest >= 0 && dest < n, err)) continue;
         if constexpr (HAS_PC) {
             emit(dest, key, s_pa[q], s_pb[q], s_pc[q]);
         } else if constexpr (emit_wants_neighbours<Emit>::value) {
@@ -239,7 +242,7 @@ struct EmitArrays3 {
 // hist: NB * ntiles uint32; offsets: NB * ntiles + 1 int64; partials: scan_partials_count(NB * ntiles) int64
 template <int BITS, typename PB, bool HAS_PC, typename Emit>
 inline cudaError_t radix_pass_impl(const uint32_t* keys, const uint32_t* pa, const PB* pb, const uint32_t* pc, int64_t n, int shift,
-                                   uint32_t* hist, int64_t* offsets, int64_t* partials, Emit emit, cudaStream_t st) {
+                                   uint32_t* hist, int64_t* offsets, int64_t* partials, Emit emit, uint32_t* err, cudaStream_t st) {
     constexpr int NB = 1 << BITS;
     const int64_t nt = radix_tiles(n);
     if (nt == 0) return cudaSuccess;
@@ -250,22 +253,22 @@ inline cudaError_t radix_pass_impl(const uint32_t* keys, const uint32_t* pa, con
     const size_t smem = RadixSmem<BITS, PB, HAS_PC>::bytes();
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<(unsigned)nt, RX_THREADS, smem, st>>>(keys, pa, pb, pc, n, shift, offsets, nt, emit);
+    kern<<<(unsigned)nt, RX_THREADS, smem, st>>>(keys, pa, pb, pc, n, shift, offsets, nt, emit, err);
     note_launches(2);
     return cudaGetLastError();
 }
 
 template <int BITS, typename PB, typename Emit>
 inline cudaError_t radix_pass(const uint32_t* keys, const uint32_t* pa, const PB* pb, int64_t n, int shift, uint32_t* hist,
-                              int64_t* offsets, int64_t* partials, Emit emit, cudaStream_t st) {
-    return radix_pass_impl<BITS, PB, false>(keys, pa, pb, nullptr, n, shift, hist, offsets, partials, emit, st);
+                              int64_t* offsets, int64_t* partials, Emit emit, uint32_t* err, cudaStream_t st) {
+    return radix_pass_impl<BITS, PB, false>(keys, pa, pb, nullptr, n, shift, hist, offsets, partials, emit, err, st);
 }
 
 // the same with a third 32-bit payload (pc == nullptr: the element's own index)
 template <int BITS, typename PB, typename Emit>
 inline cudaError_t radix_pass3(const uint32_t* keys, const uint32_t* pa, const PB* pb, const uint32_t* pc, int64_t n, int shift,
-                               uint32_t* hist, int64_t* offsets, int64_t* partials, Emit emit, cudaStream_t st) {
-    return radix_pass_impl<BITS, PB, true>(keys, pa, pb, pc, n, shift, hist, offsets, partials, emit, st);
+                               uint32_t* hist, int64_t* offsets, int64_t* partials, Emit emit, uint32_t* err, cudaStream_t st) {
+    return radix_pass_impl<BITS, PB, true>(keys, pa, pb, pc, n, shift, hist, offsets, partials, emit, err, st);
 }
 
 inline int bits_for(uint64_t max_value) {

@@ -77,6 +77,8 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     const int64_t p0 = P.rowptr[i];
     const uint32_t deg = (uint32_t)(P.rowptr[i + 1] - p0);
     const int64_t out_base = NUMERIC ? c_rowptr[rloc] : 0;
+    const int64_t out_end = NUMERIC ? c_rowptr[rloc + 1] : 0;  // bounds-checked build: no write at or past it
+    (void)out_end;
     uint32_t total_cnt = 0;
 
     // A row whose range fits one chunk and that holds a column present in every candidate row
@@ -97,10 +99,11 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
         constexpr int WHAT = decltype(what)::value;
         constexpr bool DENSE = decltype(dense_tag)::value;
         if (WHAT == CTA_SETBITS) {
-            atomicOr(&bits[rel >> 5], 1u << (rel & 31));
+            if (SPSYRK_IN_RANGE((rel >> 5) < cw, P.err)) atomicOr(&bits[rel >> 5], 1u << (rel & 31));
         } else {
+            if (!SPSYRK_IN_RANGE(DENSE || (rel >> 5) < cw, P.err)) return;
             const uint32_t slot = (DENSE ? rel : rank[rel >> 5] + __popc(bits[rel >> 5] & ((1u << (rel & 31)) - 1u))) - s0;
-            atomicAdd(&acc[slot], acc_mul(a, v));
+            if (SPSYRK_IN_RANGE(slot < tile_slots, P.err)) atomicAdd(&acc[slot], acc_mul(a, v));
         }
     };
 
@@ -250,14 +253,15 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
         if (NUMERIC) {
             const int64_t ob = out_base + total_cnt;
             if (dense) {
-                for (uint32_t t = tid; t < tot; t += THREADS) c_colidx[ob + t] = (int32_t)(c0 + t);
+                for (uint32_t t = tid; t < tot; t += THREADS)
+                    if (SPSYRK_IN_RANGE(ob + t < out_end, P.err)) c_colidx[ob + t] = (int32_t)(c0 + t);
             } else {
                 // column ids straight from the bitmap
                 for (uint32_t w = tid; w < cwa; w += THREADS) {
                     uint32_t b = bits[w], r = rank[w];
                     while (b) {
                         const int bit = __ffs(b) - 1;
-                        c_colidx[ob + r] = (int32_t)(c0 + (w << 5) + bit);
+                        if (SPSYRK_IN_RANGE(ob + r < out_end, P.err)) c_colidx[ob + r] = (int32_t)(c0 + (w << 5) + bit);
                         ++r;
                         b &= b - 1;
                     }
@@ -298,7 +302,8 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                 const bool resume = s0 > 0 && deg <= THREADS;
                 if (dense) for_each_product(ACC, IS_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
                 else for_each_product(ACC, NOT_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
-                for (uint32_t t = tid; t < s1 - s0; t += THREADS) c_vals[ob + s0 + t] = (V)(GLOBAL_ACC ? __ldcg(acc + t) : acc[t]);
+                for (uint32_t t = tid; t < s1 - s0; t += THREADS)
+                    if (SPSYRK_IN_RANGE(ob + s0 + t < out_end, P.err)) c_vals[ob + s0 + t] = (V)(GLOBAL_ACC ? __ldcg(acc + t) : acc[t]);
                 __syncthreads();
             }
         }

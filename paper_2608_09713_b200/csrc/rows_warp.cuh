@@ -181,7 +181,7 @@ numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows, con
             const uint32_t slot = t.y + e0;
 #pragma unroll
             for (uint32_t e = 0; e < 4; ++e) {
-                if (e < left) {
+                if (e < left && SPSYRK_IN_RANGE(slot + e < (uint32_t)N, P.err)) {
                     cp_async<sizeof(Rec)>(buf + slot + e, src + e);
                     own[slot + e] = (uint8_t)s;
                 }
@@ -325,6 +325,12 @@ numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows, con
             ++total;
         }
         __syncwarp();
+#ifdef SPSYRK_CHECKED
+        {
+            const int64_t room = h_n.z ? c_rowptr[h_n.x + 1] - ob_n : 0;  // the row's entries counted by the symbolic pass
+            if (!SPSYRK_IN_RANGE((int64_t)total <= room && total <= NP - 1, P.err)) total = 0;
+        }
+#endif
         for (int o = gl; o < total; o += G) {
             c_colidx[ob_n + o] = (int32_t)o_j[o + (o >> 3)];
             c_vals[ob_n + o] = o_v[o + (o >> 3)];
@@ -423,6 +429,7 @@ __global__ void __launch_bounds__(symbolic_warps(N) * 32) symbolic_warp_kernel(P
             const uint32_t s = last_not_above(s_first, c);
             const uint4 t = s_tab[s];
             const uint32_t e0 = (c - t.w) * 4u;
+            if (!SPSYRK_IN_RANGE(4 * c + 3 < (uint32_t)NS, P.err)) continue;
             cp_async<16>(buf + 4 * c, P.at_row + t.x + e0);
             // entries e0 .. e0 + 3 of the aligned run; the prefix is [lead, lead + items)
             uint32_t mk = 0;
@@ -596,6 +603,10 @@ symbolic_sort_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_
             const uint4 t = s_tab[s];
             const uint32_t e0 = (c - t.w) * 4u;
             const uint32_t lead = t.y & 0xffu, off = t.y >> 8;
+            if (!SPSYRK_IN_RANGE(4 * c + 3 < (uint32_t)NS && off + e0 + 3u - lead < (uint32_t)N + 3u, P.err)) {
+                meta[c] = 0;
+                continue;
+            }
             cp_async<16>(buf + 4 * c, P.at_row + t.x + e0);
             uint32_t mk = 0;
 #pragma unroll
@@ -630,10 +641,11 @@ symbolic_sort_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_
                 const uint4 q = buf4[c];
                 const uint32_t mt = meta[c];
                 const int tb = (int)(mt >> 4) - 3;
-                if (mt & 1u) s_jd[tb] = q.x;
-                if (mt & 2u) s_jd[tb + 1] = q.y;
-                if (mt & 4u) s_jd[tb + 2] = q.z;
-                if (mt & 8u) s_jd[tb + 3] = q.w;
+                if (!SPSYRK_IN_RANGE(tb + 3 >= 0 && tb < N, P.err)) continue;
+                if ((mt & 1u) && SPSYRK_IN_RANGE(tb >= 0, P.err)) s_jd[tb] = q.x;
+                if ((mt & 2u) && SPSYRK_IN_RANGE(tb + 1 >= 0 && tb + 1 < N, P.err)) s_jd[tb + 1] = q.y;
+                if ((mt & 4u) && SPSYRK_IN_RANGE(tb + 2 >= 0 && tb + 2 < N, P.err)) s_jd[tb + 2] = q.z;
+                if ((mt & 8u) && SPSYRK_IN_RANGE(tb + 3 < N, P.err)) s_jd[tb + 3] = q.w;
             }
         }
         __syncwarp();
@@ -788,7 +800,7 @@ numeric_map_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_t*
             const uint32_t slot = t.y + e0;
 #pragma unroll
             for (uint32_t e = 0; e < 4; ++e) {
-                if (e < left) {
+                if (e < left && SPSYRK_IN_RANGE(slot + e < (uint32_t)N, P.err)) {
                     cp_async<sizeof(Rec)>(buf + slot + e, src + e);
                     own[slot + e] = (uint8_t)s;
                 }
@@ -839,7 +851,9 @@ numeric_map_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_t*
                 prod[r] = acc_mul(a, (Acc)rc.v);
                 word[r] = mw[t];
                 const uint32_t slot = word[r] & ((1u << MAP_SLOT_BITS) - 1u);
-                if ((word[r] >> MAP_SLOT_BITS) == 0) {
+                if (!SPSYRK_IN_RANGE(slot < (uint32_t)N, P.err)) {
+                    word[r] = 0xffffffffu;
+                } else if ((word[r] >> MAP_SLOT_BITS) == 0) {
                     o_j[slot] = (uint32_t)rc.j;
                     o_v[slot] = prod[r];
                 } else {
@@ -869,7 +883,8 @@ numeric_map_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_t*
             }
         }
         int total = (int)(oe_n - ob_n);
-        if (DIAG && h_n.z > 0 && gl == 0) {
+        if (!SPSYRK_IN_RANGE(total >= 0 && total <= N + (DIAG ? 1 : 0), P.err)) total = 0;
+        if (DIAG && h_n.z > 0 && total > 0 && gl == 0) {
             o_j[total - 1] = (uint32_t)P.r0 + h_n.x;
             o_v[total - 1] = diag;
         }

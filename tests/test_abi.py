@@ -33,6 +33,13 @@ def test_every_declared_symbol_is_exported(lib):
         assert hasattr(lib, name), f"{name} is declared in spsyrk.h but not exported"
 
 
+def test_bounds_checked_build_exports_the_same_symbols():
+    from paper_2608_09713_b200 import build
+    checked = ctypes.CDLL(build.build_cuda(checked=True))
+    for name in declared_functions():
+        assert hasattr(checked, name), f"{name} is missing from the bounds-checked build"
+
+
 def test_status_strings(lib):
     lib.spsyrk_status_string.restype = ctypes.c_char_p
     seen = {lib.spsyrk_status_string(i) for i in range(9)}

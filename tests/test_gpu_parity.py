@@ -588,6 +588,13 @@ def test_permute_edge_cases(B):
     bad[0] = a.m
     with pytest.raises(B.SpsyrkError):
         B.spsyrk_permute(a.m, a.n, *d, bad)
+    # row pointers that leave [0, nnz] or do not end at nnz are rejected before any entry is moved by them
+    for where, value in ((a.m, a.nnz + 5), (a.m, a.nnz - 1), (0, 1), (7, a.nnz + 1000)):
+        badp = d[0].clone()
+        badp[where] = value
+        with pytest.raises(B.SpsyrkError) as ei:
+            B.spsyrk_permute(a.m, a.n, badp, d[1], d[2], ident)
+        assert ei.value.status == 2
     # no rows, no entries
     e = (torch.zeros(1, dtype=torch.int64, device="cuda"), torch.zeros(0, dtype=torch.int32, device="cuda"),
          torch.zeros(0, dtype=torch.float64, device="cuda"))
