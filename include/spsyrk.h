@@ -353,6 +353,12 @@ spsyrk_status_t spsyrk_plan_buffers(spsyrk_plan_t plan, const int64_t **d_colptr
  * spsyrk_launch_count       : kernels launched by this library in this process so far.
  */
 spsyrk_status_t spsyrk_plan_enable_timing(spsyrk_plan_t plan);
+/* spsyrk_mirror_enable_timing(1): from now on the fill step of spsyrk_mirror on 8-byte values records
+ *     CUDA events around each of its sorting passes (process-wide switch, not thread-safe; 0 turns it off).
+ * spsyrk_mirror_timings: *passes = sorting passes of the last such fill (at most 4) and their device
+ *     milliseconds (histogram, scan and scatter of the pass); waits for those events. */
+spsyrk_status_t spsyrk_mirror_enable_timing(int on);
+spsyrk_status_t spsyrk_mirror_timings(int *passes, float pass_ms[4]);
 spsyrk_status_t spsyrk_plan_timings(spsyrk_plan_t plan, float symbolic_ms[8], float numeric_ms[8]);
 int64_t spsyrk_launch_count(void);
 

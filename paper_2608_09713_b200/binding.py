@@ -67,6 +67,10 @@ _lib.spsyrk_status_string.restype = ctypes.c_char_p
 _lib.spsyrk_host_tril.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _vp, _vp, _vp, _int, _int, _vp, _i64p, _vp, _vp]
 _lib.spsyrk_plan_enable_timing.argtypes = [_vp]
 _lib.spsyrk_plan_timings.argtypes = [_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+_lib.spsyrk_mirror_enable_timing.argtypes = [_int]
+_lib.spsyrk_mirror_enable_timing.restype = _int
+_lib.spsyrk_mirror_timings.argtypes = [ctypes.POINTER(_int), ctypes.POINTER(ctypes.c_float)]
+_lib.spsyrk_mirror_timings.restype = _int
 _lib.spsyrk_launch_count.argtypes = []
 _lib.spsyrk_launch_count.restype = ctypes.c_int64
 for _name in ("spsyrk_plan_enable_timing", "spsyrk_plan_timings"):
@@ -222,6 +226,18 @@ def spsyrk_plan_timings(plan: Plan):
     num = (ctypes.c_float * NCLASS)()
     _check(_lib.spsyrk_plan_timings(plan._h, sym, num), "spsyrk_plan_timings")
     return list(sym), list(num)
+
+
+def spsyrk_mirror_enable_timing(on: bool = True):
+    _check(_lib.spsyrk_mirror_enable_timing(1 if on else 0), "spsyrk_mirror_enable_timing")
+
+
+def spsyrk_mirror_timings():
+    """Device milliseconds of the sorting passes of the last spsyrk_mirror fill on 8-byte values."""
+    n = _int(0)
+    ms = (ctypes.c_float * 4)()
+    _check(_lib.spsyrk_mirror_timings(ctypes.byref(n), ms), "spsyrk_mirror_timings")
+    return [float(ms[i]) for i in range(n.value)]
 
 
 def spsyrk_launch_count() -> int:

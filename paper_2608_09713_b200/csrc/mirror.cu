@@ -349,6 +349,12 @@ cudaError_t launch_mirror_pass(const MirrorPassArgs& a, int64_t n, int shift, co
     return cudaGetLastError();
 }
 
+// Measurement aid: CUDA events around every radix pass (histogram + scan + scatter) of the last record-based fill.
+constexpr int MIRROR_MAX_PASSES = 4;
+bool g_mirror_timing = false;
+cudaEvent_t g_mirror_ev[MIRROR_MAX_PASSES + 1];
+int g_mirror_passes = 0;
+
 // 8-byte values: records, the first pass straight from C_L
 spsyrk_status_t mirror_fill_rec(const MirrorWs& w, int64_t m, int64_t nnz_l, const int64_t* l_rowptr, const int32_t* l_colidx,
                                 const void* l_vals, int64_t* f_rowptr, int32_t* f_colidx, void* f_vals, cudaStream_t st) {
@@ -375,9 +381,11 @@ spsyrk_status_t mirror_fill_rec(const MirrorWs& w, int64_t m, int64_t nnz_l, con
         a.l_rowptr = l_rowptr; a.l_colidx = l_colidx; a.l_vals = lv; a.m = m; a.tile_rows = w.tile_rows;
         a.fbase = w.fbase; a.f_colidx = f_colidx; a.f_vals = fv; a.seg_start = w.seg_start; a.seg_end = w.seg_end;
         a.dtotal = w.dcount + m; a.err = w.err;
+        g_mirror_passes = 0;
         for (int p = 0; p < npass; ++p) {
             const bool first = p == 0, last = p == npass - 1;
             const bool to_a = (p % 2) == 0;
+            if (g_mirror_timing && p < MIRROR_MAX_PASSES) cudaEventRecord(g_mirror_ev[p], st);
             const unsigned hb = (unsigned)((nt + MR_HIST_TILES - 1) / MR_HIST_TILES);
             if (first) mirror_hist_key_kernel<BITS><<<hb, MR_THREADS, 0, st>>>(reinterpret_cast<const uint32_t*>(l_colidx), nnz_l, 0, w.hist, nt);
             else radix_hist_u8_kernel<BITS><<<hb, MR_THREADS, 0, st>>>(to_a ? w.dig_b : w.dig_a, nnz_l, w.hist, nt);
@@ -392,6 +400,10 @@ spsyrk_status_t mirror_fill_rec(const MirrorWs& w, int64_t m, int64_t nnz_l, con
             else if (last) e = launch_mirror_pass<false, true>(a, nnz_l, p * BITS, w.offsets, nt, st);
             else e = launch_mirror_pass<false, false>(a, nnz_l, p * BITS, w.offsets, nt, st);
             SPSYRK_CUDA_TRY(e);
+            if (g_mirror_timing && p < MIRROR_MAX_PASSES) {
+                cudaEventRecord(g_mirror_ev[p + 1], st);
+                g_mirror_passes = p + 1;
+            }
         }
     }
     if (m > 0) {
@@ -467,6 +479,28 @@ extern "C" spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_
     }
 }
 
+
+extern "C" spsyrk_status_t spsyrk_mirror_enable_timing(int on) {
+    if (on && !g_mirror_timing) {
+        for (int i = 0; i <= MIRROR_MAX_PASSES; ++i) SPSYRK_CUDA_TRY(cudaEventCreate(&g_mirror_ev[i]));
+        g_mirror_passes = 0;
+    } else if (!on && g_mirror_timing) {
+        for (int i = 0; i <= MIRROR_MAX_PASSES; ++i) cudaEventDestroy(g_mirror_ev[i]);
+    }
+    g_mirror_timing = on != 0;
+    return SPSYRK_OK;
+}
+
+extern "C" spsyrk_status_t spsyrk_mirror_timings(int* passes, float pass_ms[4]) {
+    if (!passes || !pass_ms || !g_mirror_timing) return SPSYRK_ERR_INVALID_ARG;
+    *passes = g_mirror_passes;
+    for (int p = 0; p < g_mirror_passes; ++p) {
+        pass_ms[p] = 0.f;
+        SPSYRK_CUDA_TRY(cudaEventSynchronize(g_mirror_ev[p + 1]));
+        SPSYRK_CUDA_TRY(cudaEventElapsedTime(&pass_ms[p], g_mirror_ev[p], g_mirror_ev[p + 1]));
+    }
+    return SPSYRK_OK;
+}
 
 // ------------------------------------------------------------------------------------------
 // Allocation-free computation of F's row pointers and entry count (what steps 2 and 3 of

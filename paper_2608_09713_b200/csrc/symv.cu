@@ -59,49 +59,35 @@ spsyrk_status_t symv_typed(int64_t m, int64_t nnz_l, const int64_t* l_rowptr, co
 
 namespace {
 
-// Y = C_L X + (X^T C_L)^T - D X for a dense row-major X (m x p), columns in chunks of PC: G lanes share a
-// row of C_L; for every stored entry (r, j, v) a lane adds v * X[j, c0..c0+PC) to its partial row of Y
-// (registers) and, when j != r, v * X[r, c0..c0+PC) to row j of Y (atomic adds): the diagonal is counted
-// once and C_L^T is never formed.  The rows of X are read as contiguous pieces of PC values.
-template <typename V, int G, int PC>
+// Y = C_L X + (X^T C_L)^T - D X for a dense row-major X (m x p), columns in chunks of PC = 8: one warp per row
+// of C_L, lane = (entry slot e = lane / 8, column c = lane % 8), so a warp instruction handles four stored
+// entries times eight columns.  For entry (r, j, v) lane (e, c) adds v * X[j, c0 + c] to its partial of
+// Y[r, c0 + c] (registers) and, when j != r, v * X[r, c0 + c] to Y[j, c0 + c] with an atomic add: the eight
+// adds of one entry fall into one 64-byte piece of Y (one or two sectors), which the memory system
+// handles together, instead of eight separate requests.  The diagonal is counted once and C_L^T is never formed.
+template <typename V, int PC>
 __global__ void __launch_bounds__(256) symm_kernel(int64_t m, int64_t p, int64_t c0, const int64_t* __restrict__ l_rowptr,
                                                    const int32_t* __restrict__ l_colidx, const V* __restrict__ l_vals,
                                                    const V* __restrict__ x, V* __restrict__ y) {
-    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
-    const int gl = threadIdx.x & (G - 1);
-    const int pc = (int)min((int64_t)PC, p - c0);  // columns of this chunk
-    V acc[PC], xr[PC];
-#pragma unroll
-    for (int c = 0; c < PC; ++c) { acc[c] = V(0); xr[c] = V(0); }
-    if (r < m) {
-#pragma unroll
-        for (int c = 0; c < PC; ++c)
-            if (c < pc) xr[c] = x[r * p + c0 + c];
-        const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
-        for (int64_t q = p0 + gl; q < p1; q += G) {
-            const int64_t j = l_colidx[q];
-            const V v = l_vals[q];
-            const V* xj = x + j * p + c0;
-            V* yj = y + j * p + c0;
-#pragma unroll
-            for (int c = 0; c < PC; ++c) {
-                if (c < pc) {
-                    acc[c] += v * xj[c];
-                    if (j != r) atomicAdd(&yj[c], v * xr[c]);
-                }
-            }
+    static_assert(PC == 8, "lane layout");
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = lane_id(), c = lane & 7, e = lane >> 3;
+    if (r >= m) return;  // warp-uniform
+    const bool col_on = c0 + c < p;
+    const V xr = col_on ? x[r * p + c0 + c] : V(0);
+    V acc = V(0);
+    const int64_t p0 = l_rowptr[r], p1 = l_rowptr[r + 1];
+    for (int64_t q = p0 + e; q < p1; q += 4) {
+        const int64_t j = l_colidx[q];
+        const V v = l_vals[q];
+        if (col_on) {
+            acc += v * x[j * p + c0 + c];
+            if (j != r) atomicAdd(&y[j * p + c0 + c], v * xr);
         }
     }
-#pragma unroll
-    for (int c = 0; c < PC; ++c) {
-#pragma unroll
-        for (int o = G / 2; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(FULL_MASK, acc[c], o);
-    }
-    if (r < m && gl == 0) {
-#pragma unroll
-        for (int c = 0; c < PC; ++c)
-            if (c < pc) atomicAdd(&y[r * p + c0 + c], acc[c]);
-    }
+    acc += __shfl_xor_sync(FULL_MASK, acc, 8);
+    acc += __shfl_xor_sync(FULL_MASK, acc, 16);
+    if (e == 0 && col_on) atomicAdd(&y[r * p + c0 + c], acc);
 }
 
 template <typename V>
@@ -113,14 +99,7 @@ spsyrk_status_t symm_typed(int64_t m, int64_t p, int64_t nnz_l, const int64_t* l
     V* yv = static_cast<V*>(y);
     constexpr int PC = 8;
     for (int64_t c0 = 0; c0 < p; c0 += PC) {
-#define SYMM(G) symm_kernel<V, G, PC><<<(unsigned)((m * G + 255) / 256), 256, 0, st>>>(m, p, c0, l_rowptr, l_colidx, lv, xv, yv)
-        switch (group_width(nnz_l, m)) {
-            case 4: SYMM(4); break;
-            case 8: SYMM(8); break;
-            case 16: SYMM(16); break;
-            default: SYMM(32); break;
-        }
-#undef SYMM
+        symm_kernel<V, PC><<<(unsigned)((m * 32 + 255) / 256), 256, 0, st>>>(m, p, c0, l_rowptr, l_colidx, lv, xv, yv);
         note_launches(1);
     }
     SPSYRK_CUDA_TRY(cudaGetLastError());
