@@ -293,6 +293,8 @@ def measure_workload(a, args, steps, warmup, world, rank, local, headline, dist=
             B.spsyrk_plan_set_rows(plan, *S.rank_rows(B.spsyrk_plan_partition(plan, world), rank))
         if "map" in buf:
             B.spsyrk_plan_lend_map(plan, buf["map"])
+        if is_int and not args.separate_jaccard:
+            B.spsyrk_plan_set_jaccard(plan, buf["jac"])  # the numeric pass writes the similarities with the counts
         marks.append(ev())
         c_rowptr, c_colidx, c_vals = buf["c_rowptr"], buf["c_colidx"], buf["c_vals"]
         nnz = B.spsyrk_symbolic(plan, c_rowptr)
@@ -306,7 +308,7 @@ def measure_workload(a, args, steps, warmup, world, rank, local, headline, dist=
             f = B.spsyrk_mirror(a.m, c_rowptr, c_colidx[:nnz], c_vals[:nnz], workspace=buf["mirror_ws"], out=buf["f"])
             nnz_f = f[1].numel()
         marks.append(ev())
-        if is_int:
+        if is_int and args.separate_jaccard:
             B.spsyrk_jaccard(a.m, 0, a.m, d_rowptr, c_rowptr, c_colidx[:nnz], c_vals[:nnz], out=buf["jac"])
         marks.append(ev())
         if do_mirror and sv == 8 and timing:
@@ -374,7 +376,7 @@ def measure_workload(a, args, steps, warmup, world, rank, local, headline, dist=
 
     out = {"value": value, "ms_per_step": ms_per_step, "dtype": dname, "scaling": "strong" if shard else "weak",
            "config": {"workload": a.name, "m": a.m, "n": a.n, "nnz_a": a.nnz, "multiply_adds": work_total, "nnz_c_l": nnz_c,
-                      "nnz_full": nnz_f, "step": "plan+symbolic+numeric" + ("+mirror" if do_mirror else "") + ("+jaccard" if is_int else ""),
+                      "nnz_full": nnz_f, "step": "plan+symbolic+numeric" + ("+mirror" if do_mirror else "") + (("+jaccard" if args.separate_jaccard else " (Jaccard fused into numeric)") if is_int else ""),
                       "l2_policy": "inputs_larger_than_l2" if a.nnz * (4 + sv) + nnz_c * (4 + sv) > 126e6 else "l2_flushed_by_the_other_phases",
                       "item_map": "map" in buf, "parallelism": f"rows x{world}" if shard else f"replicas x{world}"},
            "nnz_per_s": whole_job_rate(nnz_c, 1 if shard else world, ms_per_step), "phases_ms": phases,
@@ -744,6 +746,7 @@ def main():
     ap.add_argument("--no-full", action="store_true")
     ap.add_argument("--no-map", action="store_true", help="do not lend the item map: symbolic counts with hash sets, numeric sorts")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--separate-jaccard", action="store_true", help="int32 workloads: Jaccard as its own pass over the counts instead of fused into numeric")
     ap.add_argument("--no-others", action="store_true", help="headline workload only (skip the shorter runs of configurations 1-4)")
     ap.add_argument("--no-verify", action="store_true", help="skip the comparison of sampled output rows with the oracle")
     ap.add_argument("--rmat-noperm", action="store_true", help="with --rmat-scale: skip the random relabelling (load-balance study)")

@@ -327,6 +327,15 @@ spsyrk_status_t spsyrk_jaccard(int64_t m, int64_t row_begin, int64_t rows,
                                float *d_jaccard, void *cuda_stream);
 
 /*
+ * spsyrk_plan_set_jaccard - fuse the Jaccard normalisation into spsyrk_numeric: while a row's counts are
+ * written, J_ij = c_ij / (|a_i| + |a_j| - c_ij) is written to d_jaccard at the same offsets as d_c_vals
+ * (nnz entries of float; same formula and rounding as spsyrk_jaccard, so the two agree bit for bit), and
+ * the counts are not read again.  Only for I32 plans; d_jaccard == NULL switches it off.  The buffer is
+ * caller-owned and must be valid during every later spsyrk_numeric call.  Errors: INVALID_ARG.
+ */
+spsyrk_status_t spsyrk_plan_set_jaccard(spsyrk_plan_t plan, float *d_jaccard);
+
+/*
  * spsyrk_plan_stats - host-side facts about a plan.
  *   work_total    multiply-adds the plan's rows will perform (sum of w[i])
  *   class_rows[8] rows per class: 0 empty, 1..5 warp classes (w <= 32, 64, 128, 256, 512),

@@ -40,6 +40,8 @@ _lib.spsyrk_plan_set_rows.argtypes = [_vp, _i64, _i64, _vp]
 _lib.spsyrk_plan_set_block.argtypes = [_vp, _i64, _i64, _i64, _i64, _vp]
 _lib.spsyrk_plan_set_block.restype = _int
 _lib.spsyrk_symbolic.argtypes = [_vp, _vp, _i64p, _vp]
+_lib.spsyrk_plan_set_jaccard.argtypes = [_vp, _vp]
+_lib.spsyrk_plan_set_jaccard.restype = _int
 _lib.spsyrk_plan_map_bytes.argtypes = [_vp, _szp]
 _lib.spsyrk_plan_map_bytes.restype = _int
 _lib.spsyrk_plan_lend_map.argtypes = [_vp, _vp, ctypes.c_size_t]
@@ -189,6 +191,16 @@ def spsyrk_plan_lend_map(plan: Plan, item_map: torch.Tensor | None):
     _check(_lib.spsyrk_plan_lend_map(plan._h, _p(item_map), 0 if item_map is None else item_map.numel()),
            "spsyrk_plan_lend_map")
     plan._keep["map"] = item_map
+
+
+def spsyrk_plan_set_jaccard(plan: Plan, jaccard: torch.Tensor | None):
+    """From now on spsyrk_numeric also writes the Jaccard similarities into `jaccard` (float32 CUDA tensor with
+    as many entries as the product; int32 plans only); None switches the fusion off."""
+    if jaccard is not None:
+        _dev_check(jaccard)
+        assert jaccard.dtype == torch.float32
+    _check(_lib.spsyrk_plan_set_jaccard(plan._h, _p(jaccard)), "spsyrk_plan_set_jaccard")
+    plan._keep["jaccard"] = jaccard
 
 
 def spsyrk_symbolic(plan: Plan, c_rowptr: torch.Tensor, stream=None) -> int:

@@ -77,6 +77,10 @@ struct spsyrk_plan_s {
     uint32_t* row_counter;  // row dispenser of the persistent heavy-row kernel
     double* gacc;           // its global accumulator slices (GLOBAL_ACC_CTAS x gslots, 8 bytes per slot)
     uint32_t gslots;
+    uint32_t* facts;       // binary analysis (device): differs-from-one flag, heavy columns, threshold, histogram
+    uint8_t* heavy_id;
+    uint64_t* heavy_mask;
+    int32_t* adeg;
     int64_t* itemoff;      // rows + 1, class order: where the map words of a light row start
     int64_t map_items;     // map words the current row range needs
     uint16_t* map;         // caller's item map (spsyrk_plan_lend_map), or null
@@ -135,6 +139,10 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     auto row_counter = c.take<uint32_t>(1);
     auto work_prefix = c.take<int64_t>(items + 1);
     auto itemoff = c.take<int64_t>(items + 1);
+    auto heavy_id = c.take<uint8_t>(std::max<int64_t>(n, 1));
+    auto heavy_mask = c.take<uint64_t>(std::max<int64_t>(m, 1));
+    auto facts = c.take<uint32_t>(64);  // [0..2] binary analysis, [32..63] its histogram
+    auto adeg = c.take<int32_t>(std::max<int64_t>(m, 1));
     auto part_bounds = c.take<int64_t>(MAX_PARTS + 1);
     // one global accumulator slice per persistent CTA of the heavy-row numeric kernel
     const uint32_t gslots = pow2_at_least((uint64_t)std::max<int64_t>(m, 1), 1024u, ROW_CHUNK_BITS_MAX_NUMERIC);
@@ -142,6 +150,8 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     if (pl) {
         pl->row_counter = row_counter; pl->gacc = gacc; pl->gslots = gslots;
         pl->work_prefix = work_prefix; pl->part_bounds = part_bounds; pl->itemoff = itemoff;
+        pl->dev.heavy_id = heavy_id; pl->dev.heavy_mask = heavy_mask; pl->facts = facts;
+        pl->heavy_id = heavy_id; pl->heavy_mask = heavy_mask; pl->adeg = adeg; pl->dev.adeg = adeg;
         pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.at_rec = at_rec; pl->dev.desc = desc;
         pl->dev.work = work; pl->dev.err = err;
         pl->desc_full = desc; pl->desc_blk = desc_blk;
@@ -273,11 +283,15 @@ spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
         SPSYRK_CUDA_TRY(cudaMemcpyAsync(&map_items, pl->itemoff + rows, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
     }
     unsigned long long wt = 0;
+    uint32_t facts[3] = {1u, 0u, 0u};
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(facts, pl->facts, sizeof(facts), cudaMemcpyDeviceToHost, st));
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(pl->class_start, pl->class_start_dev, sizeof(pl->class_start), cudaMemcpyDeviceToHost, st));
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(&wt, pl->work_total_dev, sizeof(wt), cudaMemcpyDeviceToHost, st));
     spsyrk_status_t s = read_err(pl, st);
     pl->work_total = (int64_t)wt;
     pl->map_items = map_items;
+    pl->dev.binary = (pl->dev.nnz > 0 && facts[0] == 0) ? 1 : 0;
+    pl->dev.nheavy = pl->dev.binary ? (int32_t)std::min<uint32_t>(facts[1], 64u) : 0;
     return s;
 }
 
@@ -582,7 +596,34 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     if (s != SPSYRK_OK) return fail(s);
     s = sv == 8 ? sort_by_column<uint64_t>(pl, st) : sort_by_column<uint32_t>(pl, st);
     if (s != SPSYRK_OK) return fail(s);
-    // 3. work estimate and row binning
+    // 3. binary input: value check, heavy columns as bit masks per row
+    P.binary = 0; P.nheavy = 0; P.jaccard = nullptr;
+    PLAN_TRY(cudaMemsetAsync(pl->facts, 0, 64 * sizeof(uint32_t), st));
+    if (m > 0) {
+        row_degree_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(d_rowptr, P.m, pl->adeg);
+        note_launches(1);
+    }
+    if (nnz > 0) {
+        const unsigned cb = (unsigned)std::min<int64_t>((nnz + 255) / 256, (int64_t)pl->sm_count * 16);
+        switch (dtype) {
+            case SPSYRK_F64: binary_check_kernel<double><<<cb, 256, 0, st>>>(static_cast<const double*>(d_vals), nnz, pl->facts); break;
+            case SPSYRK_F32: binary_check_kernel<float><<<cb, 256, 0, st>>>(static_cast<const float*>(d_vals), nnz, pl->facts); break;
+            default: binary_check_kernel<int32_t><<<cb, 256, 0, st>>>(static_cast<const int32_t*>(d_vals), nnz, pl->facts); break;
+        }
+        const unsigned hb = (unsigned)std::min<int64_t>((n + 255) / 256, (int64_t)pl->sm_count * 16);
+        heavy_hist_kernel<<<hb, 256, 0, st>>>(pl->colcnt, n, pl->facts + 32);
+        heavy_threshold_kernel<<<1, 32, 0, st>>>(pl->facts + 32, pl->facts);
+        heavy_assign_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pl->colcnt, n, pl->facts, pl->heavy_id);
+        switch (group_width(nnz, m)) {
+            case 4: heavy_mask_kernel<4><<<(unsigned)((m * 4 + 255) / 256), 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
+            case 8: heavy_mask_kernel<8><<<(unsigned)((m * 8 + 255) / 256), 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
+            case 16: heavy_mask_kernel<16><<<(unsigned)((m * 16 + 255) / 256), 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
+            default: heavy_mask_kernel<32><<<(unsigned)((m * 32 + 255) / 256), 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
+        }
+        note_launches(5);
+        PLAN_TRY(cudaGetLastError());
+    }
+    // 4. work estimate and row binning (its read-back also brings the facts above)
     s = estimate_and_bin(pl, st);
     if (s != SPSYRK_OK) return fail(s);
 #undef PLAN_TRY
@@ -684,6 +725,13 @@ spsyrk_status_t spsyrk_plan_lend_map(spsyrk_plan_t plan, void* d_map, size_t byt
     plan->map_bytes = d_map ? bytes : 0;
     plan->map_filled = false;
     plan->have_symbolic = false;
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_plan_set_jaccard(spsyrk_plan_t plan, float* d_jaccard) {
+    if (!plan) return SPSYRK_ERR_INVALID_ARG;
+    if (d_jaccard && plan->dtype != SPSYRK_I32) return SPSYRK_ERR_INVALID_ARG;
+    plan->dev.jaccard = d_jaccard;
     return SPSYRK_OK;
 }
 

@@ -93,6 +93,11 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
         if (tid == 0) cnt[rloc] = (int32_t)U;
         return;
     }
+    // Binary input: a partial product is 1.  In a dense row the heavy columns' share of every count comes
+    // from the per-row bit masks (one population count per entry), and their lists are not walked.
+    const bool binary = P.binary != 0;
+    const bool use_masks = NUMERIC && dense && binary && P.nheavy > 0;
+    const unsigned long long mask_i = use_masks ? P.heavy_mask[i] : 0ull;
 
     // One partial product: set its bit, or add it into its slot.
     auto apply = [&](auto what, auto dense_tag, uint32_t rel, Acc a, Acc v, uint32_t s0) {
@@ -123,7 +128,8 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
             Acc a = Acc(0);
             if (tid == 0) s_nlong = 0;
             if (b0 + tid < deg) {
-                const uint2 d = P.desc[p0 + b0 + tid];
+                uint2 d = P.desc[p0 + b0 + tid];
+                if (WHAT == CTA_ACCUM && use_masks && P.heavy_id[P.colidx[p0 + b0 + tid]] != 0xff) d.y = 0;  // counted through the masks
                 if (whole) {
                     substart = d.x;
                     sublen = d.y;
@@ -135,7 +141,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     substart = d.x + a0;
                     sublen = a1 - a0;
                 }
-                if (WHAT == CTA_ACCUM) a = (Acc) static_cast<const V*>(P.vals)[p0 + b0 + tid];
+                if (WHAT == CTA_ACCUM) a = binary ? Acc(1) : (Acc) static_cast<const V*>(P.vals)[p0 + b0 + tid];
             }
             const bool is_long = sublen >= LONG_LIST;
             uint32_t T;
@@ -191,7 +197,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                             val[u] = Acc(0);
                             if (q[u] != 0xffffffffu) {
                                 rel[u] = (uint32_t)P.at_row[q[u]] - c0;
-                                if (WHAT == CTA_ACCUM) val[u] = (Acc) static_cast<const V*>(P.at_val)[q[u]];
+                                if (WHAT == CTA_ACCUM) val[u] = binary ? Acc(1) : (Acc) static_cast<const V*>(P.at_val)[q[u]];
                             }
                         }
 #pragma unroll
@@ -215,13 +221,13 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
 #pragma unroll
                     for (int u = 0; u < UNR; ++u) {
                         rel[u] = (uint32_t)rowp[e + u * THREADS] - c0;
-                        val[u] = WHAT == CTA_ACCUM ? (Acc)valp[e + u * THREADS] : Acc(0);
+                        val[u] = (WHAT == CTA_ACCUM && !binary) ? (Acc)valp[e + u * THREADS] : Acc(1);
                     }
 #pragma unroll
                     for (int u = 0; u < UNR; ++u) apply(what, dense_tag, rel[u], fa, val[u], s0);
                 }
                 for (; e < len; e += THREADS)
-                    apply(what, dense_tag, (uint32_t)rowp[e] - c0, fa, WHAT == CTA_ACCUM ? (Acc)valp[e] : Acc(0), s0);
+                    apply(what, dense_tag, (uint32_t)rowp[e] - c0, fa, (WHAT == CTA_ACCUM && !binary) ? (Acc)valp[e] : Acc(1), s0);
             }
             __syncthreads();
         }
@@ -297,13 +303,30 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     jlo = s_sel[0];
                     jhi = s_sel[1];
                 }
-                for (uint32_t t = tid; t < s1 - s0; t += THREADS) acc[t] = Acc(0);
+                if (use_masks) {
+                    // slot t of a dense row is column c0 + s0 + t
+                    const uint64_t* mk = P.heavy_mask + c0 + s0;
+                    for (uint32_t t = tid; t < s1 - s0; t += THREADS) acc[t] = Acc(__popcll((unsigned long long)mk[t] & mask_i));
+                } else {
+                    for (uint32_t t = tid; t < s1 - s0; t += THREADS) acc[t] = Acc(0);
+                }
                 __syncthreads();
                 const bool resume = s0 > 0 && deg <= THREADS;
                 if (dense) for_each_product(ACC, IS_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
                 else for_each_product(ACC, NOT_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
-                for (uint32_t t = tid; t < s1 - s0; t += THREADS)
-                    if (SPSYRK_IN_RANGE(ob + s0 + t < out_end, P.err)) c_vals[ob + s0 + t] = (V)(GLOBAL_ACC ? __ldcg(acc + t) : acc[t]);
+                for (uint32_t t = tid; t < s1 - s0; t += THREADS) {
+                    if (!SPSYRK_IN_RANGE(ob + s0 + t < out_end, P.err)) continue;
+                    const V cv = (V)(GLOBAL_ACC ? __ldcg(acc + t) : acc[t]);
+                    c_vals[ob + s0 + t] = cv;
+                    if constexpr (std::is_same<V, int32_t>::value) {
+                        if (P.jaccard) {
+                            // J = c / (|a_i| + |a_j| - c); the column id was written above (dense rows: it is the slot's column)
+                            const int64_t j = dense ? (int64_t)(c0 + s0 + t) : (int64_t)c_colidx[ob + s0 + t];
+                            const int64_t na_j = P.adeg[j];
+                            P.jaccard[ob + s0 + t] = __fdiv_rn((float)cv, (float)((int64_t)deg + na_j - (int64_t)cv));
+                        }
+                    }
+                }
                 __syncthreads();
             }
         }

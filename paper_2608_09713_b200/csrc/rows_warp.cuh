@@ -332,8 +332,16 @@ numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows, con
         }
 #endif
         for (int o = gl; o < total; o += G) {
-            c_colidx[ob_n + o] = (int32_t)o_j[o + (o >> 3)];
-            c_vals[ob_n + o] = o_v[o + (o >> 3)];
+            const int32_t j = (int32_t)o_j[o + (o >> 3)];
+            const V cv = o_v[o + (o >> 3)];
+            c_colidx[ob_n + o] = j;
+            c_vals[ob_n + o] = cv;
+            if constexpr (std::is_same<V, int32_t>::value) {
+                if (P.jaccard) {
+                    const int64_t na_j = P.adeg[j];
+                    P.jaccard[ob_n + o] = __fdiv_rn((float)cv, (float)((int64_t)h_n.z + na_j - (int64_t)cv));
+                }
+            }
         }
         __syncwarp();  // buffer b is handed to the gathers of row n+2 in the next iteration
 
@@ -890,8 +898,16 @@ numeric_map_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_t*
         }
         __syncwarp();
         for (int o = gl; o < total; o += G) {
-            c_colidx[ob_n + o] = (int32_t)o_j[o];
-            c_vals[ob_n + o] = (V)o_v[o];
+            const int32_t j = (int32_t)o_j[o];
+            const V cv = (V)o_v[o];
+            c_colidx[ob_n + o] = j;
+            c_vals[ob_n + o] = cv;
+            if constexpr (std::is_same<V, int32_t>::value) {
+                if (P.jaccard) {
+                    const int64_t na_j = P.adeg[j];
+                    P.jaccard[ob_n + o] = __fdiv_rn((float)cv, (float)((int64_t)h_n.z + na_j - (int64_t)cv));
+                }
+            }
         }
         __syncwarp();  // the output row and buffer b are reused
 

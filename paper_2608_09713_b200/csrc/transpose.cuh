@@ -33,7 +33,95 @@ struct PlanDev {
     uint2* desc;
     int64_t* work;  // per row of the range
     uint32_t* err;
+    // Binary input (every stored value is exactly one): a partial product is 1 and an entry of the
+    // product is an intersection count.  Then the heaviest columns (at most 64, chosen by their number
+    // of entries) are also kept as one bit per row, heavy_mask[i] bit b = row i stores heavy column b, so
+    // that their share of a count is popcount(heavy_mask[i] & heavy_mask[j]) instead of one list walk each.
+    int32_t binary;               // 0 / 1, valid after the plan's analysis
+    int32_t nheavy;               // heavy columns in use (0: none)
+    const uint8_t* heavy_id;      // [n] bit number of a heavy column, 0xff otherwise
+    const uint64_t* heavy_mask;   // [m]
+    float* jaccard;               // optional: the numeric pass also writes c / (|a_i| + |a_j| - c) here (int32 values)
+    const int32_t* adeg;          // [m] stored entries per row of A (|a_i| of the Jaccard formula)
 };
+
+static __global__ void __launch_bounds__(256) row_degree_kernel(const int64_t* __restrict__ rowptr, int32_t m, int32_t* __restrict__ adeg) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < m) adeg[i] = (int32_t)(rowptr[i + 1] - rowptr[i]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Analysis of a binary matrix: value check, choice of the heavy columns, the per-row bit masks.
+// facts[0] = 1 if some stored value differs from one; facts[1] = heavy columns; facts[2] = threshold.
+// ---------------------------------------------------------------------------------------------
+template <typename V>
+static __global__ void __launch_bounds__(256) binary_check_kernel(const V* __restrict__ vals, int64_t nnz, uint32_t* __restrict__ facts) {
+    int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    bool other = false;
+    for (; p < nnz; p += stride) other |= !(vals[p] == V(1));
+    if (__any_sync(FULL_MASK, other) && lane_id() == 0) atomicOr(&facts[0], 1u);
+}
+
+// histogram of floor(log2(column length)) over the columns
+static __global__ void __launch_bounds__(256) heavy_hist_kernel(const uint32_t* __restrict__ colcnt, int64_t n, uint32_t* __restrict__ hist32) {
+    __shared__ uint32_t h[32];
+    if (threadIdx.x < 32) h[threadIdx.x] = 0;
+    __syncthreads();
+    int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (; k < n; k += stride) {
+        const uint32_t d = colcnt[k];
+        if (d >= 256u) atomicAdd(&h[31 - __clz(d)], 1u);  // lighter columns are never candidates
+    }
+    __syncthreads();
+    if (threadIdx.x < 32 && h[threadIdx.x]) atomicAdd(&hist32[threadIdx.x], h[threadIdx.x]);
+}
+
+// threshold = the smallest power of two such that at most 64 columns have that many entries or more
+static __global__ void heavy_threshold_kernel(const uint32_t* __restrict__ hist32, uint32_t* __restrict__ facts) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    uint32_t total = 0, thr = 0xffffffffu;
+    for (int b = 31; b >= 8; --b) {
+        if (total + hist32[b] > 64u) break;
+        total += hist32[b];
+        if (hist32[b]) thr = 1u << b;
+    }
+    facts[1] = 0;
+    facts[2] = facts[0] ? 0xffffffffu : thr;  // no heavy columns unless the matrix is binary
+}
+
+static __global__ void __launch_bounds__(256) heavy_assign_kernel(const uint32_t* __restrict__ colcnt, int64_t n, uint32_t* __restrict__ facts,
+                                                                 uint8_t* __restrict__ heavy_id) {
+    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= n) return;
+    uint8_t id = 0xff;
+    if (colcnt[k] >= facts[2]) {
+        const uint32_t b = atomicAdd(&facts[1], 1u);
+        if (b < 64u) id = (uint8_t)b;
+    }
+    heavy_id[k] = id;
+}
+
+template <int G>
+static __global__ void __launch_bounds__(256) heavy_mask_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ colidx, int32_t m,
+                                                               const uint32_t* __restrict__ facts, const uint8_t* __restrict__ heavy_id,
+                                                               uint64_t* __restrict__ heavy_mask) {
+    if (facts[1] == 0) return;  // no heavy column: nothing reads the masks
+    const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    const int gl = threadIdx.x & (G - 1);
+    unsigned long long mk = 0;
+    if (gid < m) {
+        const int64_t p0 = rowptr[gid], p1 = rowptr[gid + 1];
+        for (int64_t p = p0 + gl; p < p1; p += G) {
+            const uint8_t id = heavy_id[colidx[p]];
+            if (id != 0xff) mk |= 1ull << id;
+        }
+    }
+#pragma unroll
+    for (int o = G / 2; o > 0; o >>= 1) mk |= __shfl_xor_sync(FULL_MASK, mk, o);
+    if (gid < m && gl == 0) heavy_mask[gid] = mk;
+}
 
 // One entry of a column list as a record: what the light-row numeric kernel gathers (one aligned
 // asynchronous copy per entry, whatever the list's offset).

@@ -16,9 +16,8 @@ CHECKED = os.path.join(ROOT, "paper_2608_09713_b200", "libspsyrk_checked.so")
 
 
 def test_checked_build_runs_clean():
-    if not os.path.exists(CHECKED):
-        from paper_2608_09713_b200 import build
-        build.build_cuda(checked=True)
+    from paper_2608_09713_b200 import build
+    assert build.build_cuda(checked=True) == CHECKED      # rebuilt here when a source is newer than the library
     env = dict(os.environ, SPSYRK_LIBRARY=CHECKED)
     probe = subprocess.run([sys.executable, "-c", "from paper_2608_09713_b200 import binding as B; print(B.LIB_PATH)"],
                            cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)

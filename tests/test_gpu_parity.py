@@ -258,6 +258,19 @@ def test_jaccard(B):
     jac = B.spsyrk_jaccard(a.m, 0, a.m, rowptr_a, rp, ci, cv).cpu().numpy()
     exp = oracle.jaccard(0, a.m, a.rowptr, ref.rowptr, ref.colidx, oracle.to_int32(ref.vals))
     assert np.all(np.abs(jac - exp) <= 1e-5 * np.abs(exp))
+    # fused into the numeric pass: the same numbers, bit for bit, with and without the item map
+    for item_map in (False, True):
+        plan = B.spsyrk_plan(a.m, a.n, *dev(a))
+        B.spsyrk_plan_lend_map(plan, torch.empty(max(B.spsyrk_plan_map_bytes(plan), 256), dtype=torch.uint8, device="cuda") if item_map else None)
+        rp2 = torch.empty(a.m + 1, dtype=torch.int64, device="cuda")
+        nnz = B.spsyrk_symbolic(plan, rp2)
+        ci2 = torch.empty(nnz, dtype=torch.int32, device="cuda")
+        cv2 = torch.empty(nnz, dtype=torch.int32, device="cuda")
+        fused = torch.full((nnz,), -1.0, dtype=torch.float32, device="cuda")
+        B.spsyrk_plan_set_jaccard(plan, fused)
+        B.spsyrk_numeric(plan, rp2, ci2, cv2)
+        assert torch.equal(ci2, ci) and torch.equal(cv2, cv)
+        assert np.array_equal(fused.cpu().numpy(), jac)
     assert np.array_equal(jac, exp)                          # one correctly rounded division on both sides
     rows = np.repeat(np.arange(a.m), np.diff(ref.rowptr))
     assert np.all(jac[rows == ref.colidx] == 1.0)
@@ -677,6 +690,35 @@ def test_rows_with_33_nonzeros_leave_the_warp_classes(B):
     _, classes = B.spsyrk_plan_stats(plan)
     assert sum(classes[6:]) >= m // 2
     run_and_compare(B, a, 1)
+
+
+# ------------------------------------------------ binary matrices: heavy columns through bit masks
+@pytest.mark.parametrize("dtype", [np.int32, np.float64])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_binary_matrix_with_heavy_columns(B, dtype, mode):
+    """All values one, a column in every row (every output row is dense), more than 64 columns with 256 or more
+    entries (so only the heaviest go through the bit masks) and rows of every class."""
+    rng = np.random.default_rng(31)
+    m, n = 3000, 5000
+    mask = rng.random((m, n)) < 0.004
+    mask[:, 17] = True
+    for k, dens in zip(rng.choice(n, size=90, replace=False), np.linspace(0.09, 0.9, 90)):
+        mask[:, k] |= rng.random(m) < dens
+    rr, cc = np.nonzero(mask)
+    rowptr = np.zeros(m + 1, dtype=np.int64)
+    np.cumsum(np.bincount(rr, minlength=m), out=rowptr[1:])
+    a = W.CSR(m, n, rowptr, cc.astype(np.int32), np.ones(cc.size, dtype=dtype))
+    (rp, ci, cv), ref, plan = run_and_compare(B, a, mode)
+    if dtype == np.int32 and mode == 0:
+        jac = torch.empty(ci.numel(), dtype=torch.float32, device="cuda")
+        B.spsyrk_plan_set_jaccard(plan, jac)
+        B.spsyrk_numeric(plan, rp, ci, cv)
+        exp = oracle.jaccard(0, a.m, a.rowptr, ref.rowptr, ref.colidx, oracle.to_int32(ref.vals))
+        assert np.array_equal(jac.cpu().numpy(), exp)
+    # the same structure with one value that is not one: the plain path must give the plain answer
+    vals = np.ones(cc.size, dtype=dtype)
+    vals[cc.size // 2] = 3
+    run_and_compare(B, W.CSR(m, n, rowptr, cc.astype(np.int32), vals), mode)
 
 
 # ------------------------------------------------ heavy rows beyond one bitmap chunk (more than 2^20 rows)
