@@ -54,6 +54,20 @@ uint32_t pow2_at_least(uint64_t v, uint32_t lo, uint32_t hi) {
 struct spsyrk_plan_s {
     PlanDev dev;
     spsyrk_dtype_t dtype;
+    // Full-output mode over the whole column range is computed in two parts per row: the lower part (columns
+    // <= row, this object, working exactly like the lower-triangle mode) and the upper part (columns > row, the
+    // `upper` view: the rest of every column list).  The two parts of a row are sorted ranges that follow
+    // each other in the output, so each is a product of half the size and the light-row kernels see rows of
+    // half the work.  dev.mode is the column range the kernels of a view work on; user_mode what was asked for.
+    spsyrk_mode_t user_mode;
+    spsyrk_plan_s* upper;   // null in lower-triangle mode
+    bool upper_active;      // the current range is computed in two parts
+    uint2* desc_hi;         // descriptors of the upper parts (start after the row's own entry, rest of the column)
+    int32_t* cnt_tot;       // rows: entries per row, both parts
+    int64_t* hi_begin;      // rows + 1: where the upper part of every row starts in the output
+    int64_t* work_sum;      // rows: work of both parts
+    const int64_t* out_begin;  // set by spsyrk_numeric: where each row's part starts / ends in the output
+    const int64_t* out_end;
     int64_t rows_cap;
     // workspace views
     int32_t* perm;
@@ -103,7 +117,7 @@ struct spsyrk_plan_s {
 
 namespace {
 
-size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, size_t sv) {
+size_t carve(spsyrk_plan_s* pl, spsyrk_plan_s* up, void* ws, int64_t m, int64_t n, int64_t nnz, size_t sv, bool full) {
     Carver c(ws);
     const int64_t items = std::max<int64_t>(std::max(m, n), 1);
     const int64_t nb = bin_blocks(items);
@@ -147,7 +161,29 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
     // one global accumulator slice per persistent CTA of the heavy-row numeric kernel
     const uint32_t gslots = pow2_at_least((uint64_t)std::max<int64_t>(m, 1), 1024u, ROW_CHUNK_BITS_MAX_NUMERIC);
     auto gacc = c.take<double>((size_t)GLOBAL_ACC_CTAS * gslots);
+    // full-output mode: the upper view's own per-row arrays and the second descriptor array
+    uint2* desc_hi = nullptr;
+    int64_t *u_work = nullptr, *u_itemoff = nullptr, *u_class_start_dev = nullptr, *hi_begin = nullptr, *work_sum = nullptr;
+    int32_t *u_perm = nullptr, *u_cnt = nullptr, *cnt_tot = nullptr;
+    uint4* u_hdr = nullptr;
+    uint8_t* u_cls = nullptr;
+    unsigned long long* u_work_total_dev = nullptr;
+    if (full) {
+        desc_hi = c.take<uint2>(nnz);
+        u_work = c.take<int64_t>(m);
+        u_perm = c.take<int32_t>(m);
+        u_hdr = c.take<uint4>(m);
+        u_cnt = c.take<int32_t>(m);
+        u_cls = c.take<uint8_t>(items);
+        u_itemoff = c.take<int64_t>(items + 1);
+        u_class_start_dev = c.take<int64_t>(NCLASS + 1);
+        u_work_total_dev = c.take<unsigned long long>(1);
+        cnt_tot = c.take<int32_t>(m);
+        hi_begin = c.take<int64_t>(items + 1);
+        work_sum = c.take<int64_t>(m);
+    }
     if (pl) {
+        pl->desc_hi = desc_hi; pl->cnt_tot = cnt_tot; pl->hi_begin = hi_begin; pl->work_sum = work_sum;
         pl->row_counter = row_counter; pl->gacc = gacc; pl->gslots = gslots;
         pl->work_prefix = work_prefix; pl->part_bounds = part_bounds; pl->itemoff = itemoff;
         pl->dev.heavy_id = heavy_id; pl->dev.heavy_mask = heavy_mask; pl->facts = facts;
@@ -160,6 +196,14 @@ size_t carve(spsyrk_plan_s* pl, void* ws, int64_t m, int64_t n, int64_t nnz, siz
         pl->rx_pos_b = rx_pos_b; pl->rx_val_a = rx_val_a; pl->rx_val_b = rx_val_b; pl->rx_hist = rx_hist; pl->rx_offsets = rx_offsets;
         pl->blockhist = blockhist; pl->offsets = offsets; pl->partials = partials;
         pl->class_start_dev = class_start_dev; pl->work_total_dev = work_total_dev;
+        if (up) {
+            // the upper view shares everything that describes A and the scratch space; its rows are its own
+            *up = *pl;
+            up->upper = nullptr;
+            up->dev.desc = desc_hi; up->dev.work = u_work;
+            up->perm = u_perm; up->hdr = u_hdr; up->cnt = u_cnt; up->cls = u_cls; up->itemoff = u_itemoff;
+            up->class_start_dev = u_class_start_dev; up->work_total_dev = u_work_total_dev;
+        }
     }
     return (c.off + ALIGN - 1) / ALIGN * ALIGN;
 }
@@ -185,7 +229,7 @@ template <int G>
 void launch_block_desc(spsyrk_plan_s* pl, cudaStream_t st) {
     const PlanDev& P = pl->dev;
     const int64_t threads = (int64_t)(P.r1 - P.r0) * G;
-    block_desc_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P, pl->desc_full, pl->desc_blk, pl->s0, pl->s1);
+    block_desc_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P, pl->desc_full, pl->user_mode == SPSYRK_FULL ? pl->desc_hi : nullptr, pl->desc_blk, pl->s0, pl->s1);
     note_launches(1);
 }
 
@@ -222,7 +266,7 @@ spsyrk_status_t sort_by_column(spsyrk_plan_s* pl, cudaStream_t st) {
         uint32_t* dst_pos = to_a ? pl->rx_pos_a : pl->rx_pos_b;
         VB* dst_val = static_cast<VB*>(to_a ? pl->rx_val_a : pl->rx_val_b);
         if (p == npass - 1) {
-            EmitTransposeFinal<VB> emit{P};
+            EmitTransposeFinal<VB> emit{P, pl->desc_hi};
             SPSYRK_CUDA_TRY((radix_pass3<BITS, VB>(src_key, src_row, src_val, src_pos, P.nnz, p * BITS, pl->rx_hist, pl->rx_offsets,
                                                    pl->partials, emit, P.err, st)));
         } else {
@@ -238,26 +282,16 @@ spsyrk_status_t sort_by_column(spsyrk_plan_s* pl, cudaStream_t st) {
     return SPSYRK_OK;
 }
 
-// work estimate + binning of the plan's current row range; reads class sizes back (one sync)
-spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
+__global__ void add_work_kernel(const int64_t* __restrict__ a, const int64_t* __restrict__ b, int64_t rows, int64_t* __restrict__ out) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < rows) out[r] = a[r] + b[r];
+}
+
+// work estimate + binning of one view's current row range (dev.desc, dev.mode and diag are set); reads class sizes back (one sync)
+spsyrk_status_t bin_view(spsyrk_plan_s* pl, cudaStream_t st) {
     const int64_t rows = pl->dev.r1 - pl->dev.r0;
     pl->have_symbolic = false;
-    // descriptors: the transpose's own for the whole column range, else narrowed to [s0, s1)
-    if (pl->s0 <= 0 && pl->s1 >= pl->dev.m) {
-        pl->dev.desc = pl->desc_full;
-    } else {
-        pl->dev.desc = pl->desc_blk;
-        if (rows > 0 && pl->dev.nnz > 0) {
-            switch (group_width(pl->dev.nnz, pl->dev.m)) {
-                case 4: launch_block_desc<4>(pl, st); break;
-                case 8: launch_block_desc<8>(pl, st); break;
-                case 16: launch_block_desc<16>(pl, st); break;
-                default: launch_block_desc<32>(pl, st); break;
-            }
-        }
-    }
     const PlanDev& P = pl->dev;
-    pl->diag = P.mode == SPSYRK_TRIL && pl->dev.desc == pl->desc_full;
     SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->work_total_dev, 0, sizeof(unsigned long long), st));
     if (rows > 0) {
         switch (group_width(P.nnz, P.m)) {
@@ -295,7 +329,56 @@ spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
     return s;
 }
 
-bool use_map(const spsyrk_plan_s* pl) { return pl->map && pl->map_bytes >= (size_t)pl->map_items * sizeof(uint16_t); }
+// descriptors, work estimate and binning of the plan's current block of output rows and columns
+spsyrk_status_t estimate_and_bin(spsyrk_plan_s* pl, cudaStream_t st) {
+    const int64_t rows = pl->dev.r1 - pl->dev.r0;
+    const bool whole = pl->s0 <= 0 && pl->s1 >= pl->dev.m;
+    pl->upper_active = false;
+    if (whole) {
+        pl->dev.desc = pl->desc_full;
+        if (pl->user_mode == SPSYRK_FULL && pl->upper) {
+            // two parts per row: this view does the lower parts like the lower-triangle mode, the upper view the rest
+            pl->upper_active = true;
+            pl->dev.mode = SPSYRK_TRIL;
+            pl->diag = true;
+            spsyrk_status_t s = bin_view(pl, st);
+            if (s != SPSYRK_OK) return s;
+            spsyrk_plan_s* up = pl->upper;
+            up->dev.r0 = pl->dev.r0; up->dev.r1 = pl->dev.r1;
+            up->dev.mode = SPSYRK_FULL;  // the upper part of row i lies in (i, m): the kernels work on the range [0, m)
+            up->dev.desc = pl->desc_hi;
+            up->dev.jaccard = pl->dev.jaccard;
+            up->diag = false;
+            s = bin_view(up, st);
+            if (s != SPSYRK_OK) return s;
+            if (rows > 0) {
+                add_work_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(pl->dev.work, up->dev.work, rows, pl->work_sum);
+                note_launches(1);
+            }
+            return SPSYRK_OK;
+        }
+        pl->dev.mode = (int32_t)pl->user_mode;
+        pl->diag = pl->user_mode == SPSYRK_TRIL;
+        return bin_view(pl, st);
+    }
+    // a column range: descriptors narrowed to [s0, s1) (cut out of the whole column lists in full-output mode)
+    pl->dev.desc = pl->desc_blk;
+    pl->dev.mode = (int32_t)pl->user_mode;
+    pl->diag = false;
+    if (rows > 0 && pl->dev.nnz > 0) {
+        switch (group_width(pl->dev.nnz, pl->dev.m)) {
+            case 4: launch_block_desc<4>(pl, st); break;
+            case 8: launch_block_desc<8>(pl, st); break;
+            case 16: launch_block_desc<16>(pl, st); break;
+            default: launch_block_desc<32>(pl, st); break;
+        }
+    }
+    return bin_view(pl, st);
+}
+
+int64_t map_items_total(const spsyrk_plan_s* pl) { return pl->map_items + (pl->upper_active ? pl->upper->map_items : 0); }
+
+bool use_map(const spsyrk_plan_s* pl) { return pl->map && pl->map_bytes >= (size_t)map_items_total(pl) * sizeof(uint16_t); }
 
 template <int N, bool DIAG>
 spsyrk_status_t launch_symbolic_warp_d(spsyrk_plan_s* pl, int c, cudaStream_t st) {
@@ -322,7 +405,7 @@ spsyrk_status_t launch_symbolic_warp(spsyrk_plan_s* pl, int c, cudaStream_t st) 
 }
 
 template <typename V, int N, typename Key, bool DIAG>
-spsyrk_status_t launch_numeric_warp_d(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+spsyrk_status_t launch_numeric_warp_d(spsyrk_plan_s* pl, int c, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
     const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
     if (count <= 0) return SPSYRK_OK;
     constexpr int G = warp_class_group(N);
@@ -337,16 +420,16 @@ spsyrk_status_t launch_numeric_warp_d(spsyrk_plan_s* pl, int c, const int64_t* c
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
     const int64_t want = (count + ROWS - 1) / ROWS;
     const int64_t cap = (int64_t)pl->sm_count * per_sm;
-    kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, c_rowptr, c_colidx,
-                                                               static_cast<V*>(c_vals));
+    kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, pl->out_begin, pl->out_end,
+                                                               c_colidx, static_cast<V*>(c_vals));
     note_launches(1);
     return SPSYRK_OK;
 }
 
 template <typename V, int N, typename Key>
-spsyrk_status_t launch_numeric_warp(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
-    return pl->diag ? launch_numeric_warp_d<V, N, Key, true>(pl, c, c_rowptr, c_colidx, c_vals, st)
-                    : launch_numeric_warp_d<V, N, Key, false>(pl, c, c_rowptr, c_colidx, c_vals, st);
+spsyrk_status_t launch_numeric_warp(spsyrk_plan_s* pl, int c, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    return pl->diag ? launch_numeric_warp_d<V, N, Key, true>(pl, c, c_colidx, c_vals, st)
+                    : launch_numeric_warp_d<V, N, Key, false>(pl, c, c_colidx, c_vals, st);
 }
 
 template <int N, typename Key, bool DIAG>
@@ -377,7 +460,7 @@ spsyrk_status_t launch_symbolic_sort(spsyrk_plan_s* pl, int c, cudaStream_t st) 
 }
 
 template <typename V, int N, bool DIAG>
-spsyrk_status_t launch_numeric_map_d(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+spsyrk_status_t launch_numeric_map_d(spsyrk_plan_s* pl, int c, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
     const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
     if (count <= 0) return SPSYRK_OK;
     constexpr int G = warp_class_group(N);
@@ -391,15 +474,15 @@ spsyrk_status_t launch_numeric_map_d(spsyrk_plan_s* pl, int c, const int64_t* c_
     const int64_t want = (count + ROWS - 1) / ROWS;
     const int64_t cap = (int64_t)pl->sm_count * per_sm;
     kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], pl->itemoff + pl->class_start[c],
-                                                               count, pl->map, c_rowptr, c_colidx, static_cast<V*>(c_vals));
+                                                               count, pl->map, pl->out_begin, pl->out_end, c_colidx, static_cast<V*>(c_vals));
     note_launches(1);
     return SPSYRK_OK;
 }
 
 template <typename V, int N>
-spsyrk_status_t launch_numeric_map(spsyrk_plan_s* pl, int c, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
-    return pl->diag ? launch_numeric_map_d<V, N, true>(pl, c, c_rowptr, c_colidx, c_vals, st)
-                    : launch_numeric_map_d<V, N, false>(pl, c, c_rowptr, c_colidx, c_vals, st);
+spsyrk_status_t launch_numeric_map(spsyrk_plan_s* pl, int c, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    return pl->diag ? launch_numeric_map_d<V, N, true>(pl, c, c_colidx, c_vals, st)
+                    : launch_numeric_map_d<V, N, false>(pl, c, c_colidx, c_vals, st);
 }
 
 inline void mark(spsyrk_plan_s* pl, cudaEvent_t* ev, int i, cudaStream_t st) {
@@ -407,32 +490,32 @@ inline void mark(spsyrk_plan_s* pl, cudaEvent_t* ev, int i, cudaStream_t st) {
 }
 
 template <typename V>
-void launch_numeric_map_all(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+void launch_numeric_map_all(spsyrk_plan_s* pl, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
     mark(pl, pl->ev_num, 1, st);
-    launch_numeric_map<V, 32>(pl, 1, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_map<V, 32>(pl, 1, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 2, st);
-    launch_numeric_map<V, 64>(pl, 2, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_map<V, 64>(pl, 2, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 3, st);
-    launch_numeric_map<V, 128>(pl, 3, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_map<V, 128>(pl, 3, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 4, st);
-    launch_numeric_map<V, 256>(pl, 4, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_map<V, 256>(pl, 4, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 5, st);
-    launch_numeric_map<V, 512>(pl, 5, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_map<V, 512>(pl, 5, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 6, st);
 }
 
 template <typename V, typename Key>
-void launch_numeric_warp_all(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+void launch_numeric_warp_all(spsyrk_plan_s* pl, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
     mark(pl, pl->ev_num, 1, st);
-    launch_numeric_warp<V, 32, Key>(pl, 1, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 32, Key>(pl, 1, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 2, st);
-    launch_numeric_warp<V, 64, Key>(pl, 2, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 64, Key>(pl, 2, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 3, st);
-    launch_numeric_warp<V, 128, Key>(pl, 3, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 128, Key>(pl, 3, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 4, st);
-    launch_numeric_warp<V, 256, Key>(pl, 4, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 256, Key>(pl, 4, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 5, st);
-    launch_numeric_warp<V, 512, Key>(pl, 5, c_rowptr, c_colidx, c_vals, st);
+    launch_numeric_warp<V, 512, Key>(pl, 5, c_colidx, c_vals, st);
     mark(pl, pl->ev_num, 6, st);
 }
 
@@ -465,14 +548,13 @@ spsyrk_status_t launch_symbolic_cta(spsyrk_plan_s* pl, int c, cudaStream_t st) {
     auto kern = rows_cta_kernel<int32_t, THREADS, false>;
     SPSYRK_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, 0u, pl->cnt, nullptr, nullptr, nullptr,
-                                                  0u, nullptr, nullptr, 0u);
+                                                  nullptr, 0u, nullptr, nullptr, 0u);
     note_launches(1);
     return SPSYRK_OK;
 }
 
 template <typename V, int THREADS>
-spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_or_zero, const int64_t* c_rowptr, int32_t* c_colidx,
-                                   void* c_vals, cudaStream_t st) {
+spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_or_zero, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
     using Acc = typename AccOf<V>::type;
     const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
     if (count <= 0) return SPSYRK_OK;
@@ -489,8 +571,8 @@ spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_
     // rows that overflow the shared-memory tile go to the persistent variant with global accumulators
     const bool use_global = acc_slots_or_zero == 0 && pl->gslots >= cb;
     const uint32_t gslots = use_global ? pl->gslots : 0u;
-    kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, c_rowptr, c_colidx,
-                                                  static_cast<V*>(c_vals), 0u, nullptr, nullptr, gslots);
+    kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, pl->out_begin, pl->out_end,
+                                                  c_colidx, static_cast<V*>(c_vals), 0u, nullptr, nullptr, gslots);
     note_launches(1);
     if (use_global) {
         auto gkern = rows_cta_kernel<V, THREADS, true, true>;
@@ -498,8 +580,8 @@ spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_
         SPSYRK_CUDA_TRY(cudaFuncSetAttribute(gkern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gsmem));
         SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->row_counter, 0, sizeof(uint32_t), st));
         const unsigned grid = (unsigned)std::min<int64_t>(std::min<int64_t>(pl->sm_count, GLOBAL_ACC_CTAS), count);
-        gkern<<<grid, THREADS, gsmem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, c_rowptr, c_colidx,
-                                            static_cast<V*>(c_vals), (uint32_t)count, pl->row_counter,
+        gkern<<<grid, THREADS, gsmem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, pl->out_begin, pl->out_end,
+                                            c_colidx, static_cast<V*>(c_vals), (uint32_t)count, pl->row_counter,
                                             reinterpret_cast<Acc*>(pl->gacc), gslots);
         note_launches(1);
     }
@@ -507,14 +589,14 @@ spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_
 }
 
 template <typename V>
-spsyrk_status_t numeric_typed(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
-    if (pl->map_filled) launch_numeric_map_all<V>(pl, c_rowptr, c_colidx, c_vals, st);
-    else if (pl->key64) launch_numeric_warp_all<V, uint64_t>(pl, c_rowptr, c_colidx, c_vals, st);
-    else launch_numeric_warp_all<V, uint32_t>(pl, c_rowptr, c_colidx, c_vals, st);
-    spsyrk_status_t s = launch_numeric_cta<V, 256>(pl, 6, BLOCK_ACC_SLOTS, c_rowptr, c_colidx, c_vals, st);
+spsyrk_status_t numeric_typed(spsyrk_plan_s* pl, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
+    if (pl->map_filled) launch_numeric_map_all<V>(pl, c_colidx, c_vals, st);
+    else if (pl->key64) launch_numeric_warp_all<V, uint64_t>(pl, c_colidx, c_vals, st);
+    else launch_numeric_warp_all<V, uint32_t>(pl, c_colidx, c_vals, st);
+    spsyrk_status_t s = launch_numeric_cta<V, 256>(pl, 6, BLOCK_ACC_SLOTS, c_colidx, c_vals, st);
     if (s != SPSYRK_OK) return s;
     mark(pl, pl->ev_num, 7, st);
-    s = launch_numeric_cta<V, 1024>(pl, 7, 0u, c_rowptr, c_colidx, c_vals, st);
+    s = launch_numeric_cta<V, 1024>(pl, 7, 0u, c_colidx, c_vals, st);
     if (s != SPSYRK_OK) return s;
     mark(pl, pl->ev_num, 8, st);
     SPSYRK_CUDA_TRY(cudaGetLastError());
@@ -523,6 +605,43 @@ spsyrk_status_t numeric_typed(spsyrk_plan_s* pl, const int64_t* c_rowptr, int32_
 #else
     return SPSYRK_OK;
 #endif
+}
+
+__global__ void add_counts_kernel(const int32_t* __restrict__ a, const int32_t* __restrict__ b, int64_t rows, int32_t* __restrict__ out) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < rows) out[r] = a[r] + b[r];
+}
+
+__global__ void upper_begin_kernel(const int64_t* __restrict__ c_rowptr, const int32_t* __restrict__ cnt_lo, int64_t rows,
+                                   int64_t* __restrict__ hi_begin) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < rows) hi_begin[r] = c_rowptr[r] + cnt_lo[r];
+}
+
+// the per-class count kernels of one view (entries per row into its cnt array)
+spsyrk_status_t symbolic_view(spsyrk_plan_s* pl, bool with_map, cudaStream_t st) {
+    const int64_t rows = pl->dev.r1 - pl->dev.r0;
+    if (rows > 0) SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->cnt, 0, (size_t)rows * sizeof(int32_t), st));
+    pl->map_filled = false;
+    mark(pl, pl->ev_sym, 1, st);
+    if (with_map) launch_symbolic_sort<32>(pl, 1, st); else launch_symbolic_warp<32>(pl, 1, st);
+    mark(pl, pl->ev_sym, 2, st);
+    if (with_map) launch_symbolic_sort<64>(pl, 2, st); else launch_symbolic_warp<64>(pl, 2, st);
+    mark(pl, pl->ev_sym, 3, st);
+    if (with_map) launch_symbolic_sort<128>(pl, 3, st); else launch_symbolic_warp<128>(pl, 3, st);
+    mark(pl, pl->ev_sym, 4, st);
+    if (with_map) launch_symbolic_sort<256>(pl, 4, st); else launch_symbolic_warp<256>(pl, 4, st);
+    mark(pl, pl->ev_sym, 5, st);
+    if (with_map) launch_symbolic_sort<512>(pl, 5, st); else launch_symbolic_warp<512>(pl, 5, st);
+    mark(pl, pl->ev_sym, 6, st);
+    spsyrk_status_t s = launch_symbolic_cta<256>(pl, 6, st);
+    if (s != SPSYRK_OK) return s;
+    mark(pl, pl->ev_sym, 7, st);
+    s = launch_symbolic_cta<1024>(pl, 7, st);
+    if (s != SPSYRK_OK) return s;
+    mark(pl, pl->ev_sym, 8, st);
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    return SPSYRK_OK;
 }
 
 }  // namespace
@@ -539,7 +658,8 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     if (row_begin < 0 || row_end < row_begin || row_end > m) return SPSYRK_ERR_INVALID_ARG;
     if (m >= (int64_t(1) << 31) - 1 || n >= (int64_t(1) << 31) - 1 || nnz >= (int64_t(1) << 31) - 1) return SPSYRK_ERR_OVERFLOW;
     const size_t sv = dtype_size(dtype);
-    const size_t need = carve(nullptr, nullptr, m, n, nnz, sv);
+    const bool full = mode == SPSYRK_FULL;
+    const size_t need = carve(nullptr, nullptr, nullptr, m, n, nnz, sv, full);
     if (!d_workspace) {
         *workspace_bytes = need;
         return SPSYRK_OK;
@@ -556,6 +676,7 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     P.m = (int32_t)m; P.n = (int32_t)n; P.nnz = nnz; P.r0 = (int32_t)row_begin; P.r1 = (int32_t)row_end; P.mode = (int32_t)mode;
     P.rowptr = d_rowptr; P.colidx = d_colidx; P.vals = d_vals;
     pl->dtype = dtype;
+    pl->user_mode = mode;
     pl->rows_cap = m;
     pl->key64 = m > (int64_t(1) << 22);
     pl->s0 = 0;
@@ -565,9 +686,16 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
         pl->sm_count = 148;
         if (cudaGetDevice(&dev_id) == cudaSuccess) cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, dev_id);
     }
-    carve(pl, d_workspace, m, n, nnz, sv);
+    spsyrk_plan_s* up = nullptr;
+    if (full) {
+        up = new (std::nothrow) spsyrk_plan_s();
+        if (!up) { delete pl; return SPSYRK_ERR_INTERNAL; }
+    }
+    pl->upper = up;
+    carve(pl, up, d_workspace, m, n, nnz, sv, full);
+    pl->upper = up;  // (the copy into the upper view happened with a null link)
 
-    auto fail = [&](spsyrk_status_t s) { delete pl; return s; };
+    auto fail = [&](spsyrk_status_t s) { delete up; delete pl; return s; };
 #define PLAN_TRY(expr) do { if ((expr) != cudaSuccess) return fail(SPSYRK_ERR_CUDA); } while (0)
     PLAN_TRY(cudaMemsetAsync(P.err, 0, sizeof(uint32_t), st));
     if (n > 0) PLAN_TRY(cudaMemsetAsync(pl->colcnt, 0, (size_t)n * sizeof(uint32_t), st));
@@ -614,11 +742,12 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
         heavy_hist_kernel<<<hb, 256, 0, st>>>(pl->colcnt, n, pl->facts + 32);
         heavy_threshold_kernel<<<1, 32, 0, st>>>(pl->facts + 32, pl->facts);
         heavy_assign_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pl->colcnt, n, pl->facts, pl->heavy_id);
+        const unsigned mb = (unsigned)std::min<int64_t>((m * 32 + 255) / 256, (int64_t)pl->sm_count * 8);
         switch (group_width(nnz, m)) {
-            case 4: heavy_mask_kernel<4><<<(unsigned)((m * 4 + 255) / 256), 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
-            case 8: heavy_mask_kernel<8><<<(unsigned)((m * 8 + 255) / 256), 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
-            case 16: heavy_mask_kernel<16><<<(unsigned)((m * 16 + 255) / 256), 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
-            default: heavy_mask_kernel<32><<<(unsigned)((m * 32 + 255) / 256), 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
+            case 4: heavy_mask_kernel<4><<<mb, 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
+            case 8: heavy_mask_kernel<8><<<mb, 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
+            case 16: heavy_mask_kernel<16><<<mb, 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
+            default: heavy_mask_kernel<32><<<mb, 256, 0, st>>>(d_rowptr, d_colidx, P.m, pl->facts, pl->heavy_id, pl->heavy_mask); break;
         }
         note_launches(5);
         PLAN_TRY(cudaGetLastError());
@@ -639,6 +768,7 @@ spsyrk_status_t spsyrk_plan_set_block(spsyrk_plan_t plan, int64_t row_begin, int
     plan->dev.r1 = (int32_t)row_end;
     plan->s0 = (int32_t)col_begin;
     plan->s1 = (int32_t)col_end;
+    plan->have_symbolic = false;
     return estimate_and_bin(plan, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -650,10 +780,11 @@ spsyrk_status_t spsyrk_plan_set_rows(spsyrk_plan_t plan, int64_t row_begin, int6
 spsyrk_status_t spsyrk_plan_partition(spsyrk_plan_t plan, int64_t parts, int64_t* bounds, void* cuda_stream) {
     if (!plan || !bounds || parts < 1 || parts > MAX_PARTS) return SPSYRK_ERR_INVALID_ARG;
     spsyrk_plan_s* pl = plan;
-    if (pl->work_total > 0 && pl->work_total > INT64_MAX / parts) return SPSYRK_ERR_OVERFLOW;
+    const int64_t work_all = pl->work_total + (pl->upper_active ? pl->upper->work_total : 0);
+    if (work_all > 0 && work_all > INT64_MAX / parts) return SPSYRK_ERR_OVERFLOW;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int64_t rows = pl->dev.r1 - pl->dev.r0;
-    SPSYRK_CUDA_TRY(exclusive_scan_i64<int64_t>(pl->dev.work, rows, pl->work_prefix, pl->partials, st));
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<int64_t>(pl->upper_active ? pl->work_sum : pl->dev.work, rows, pl->work_prefix, pl->partials, st));
     partition_kernel<<<(unsigned)((parts + 1 + 255) / 256), 256, 0, st>>>(pl->work_prefix, rows, parts, pl->dev.r0, pl->part_bounds);
     note_launches(1);
     SPSYRK_CUDA_TRY(cudaGetLastError());
@@ -667,28 +798,28 @@ spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t* d_c_rowptr, int64_t
     spsyrk_plan_s* pl = plan;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const int64_t rows = pl->dev.r1 - pl->dev.r0;
-    if (rows > 0) SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->cnt, 0, (size_t)rows * sizeof(int32_t), st));
     const bool with_map = use_map(pl);
-    pl->map_filled = false;
-    mark(pl, pl->ev_sym, 1, st);
-    if (with_map) launch_symbolic_sort<32>(pl, 1, st); else launch_symbolic_warp<32>(pl, 1, st);
-    mark(pl, pl->ev_sym, 2, st);
-    if (with_map) launch_symbolic_sort<64>(pl, 2, st); else launch_symbolic_warp<64>(pl, 2, st);
-    mark(pl, pl->ev_sym, 3, st);
-    if (with_map) launch_symbolic_sort<128>(pl, 3, st); else launch_symbolic_warp<128>(pl, 3, st);
-    mark(pl, pl->ev_sym, 4, st);
-    if (with_map) launch_symbolic_sort<256>(pl, 4, st); else launch_symbolic_warp<256>(pl, 4, st);
-    mark(pl, pl->ev_sym, 5, st);
-    if (with_map) launch_symbolic_sort<512>(pl, 5, st); else launch_symbolic_warp<512>(pl, 5, st);
-    mark(pl, pl->ev_sym, 6, st);
-    spsyrk_status_t s = launch_symbolic_cta<256>(pl, 6, st);
+    spsyrk_status_t s = symbolic_view(pl, with_map, st);
     if (s != SPSYRK_OK) return s;
-    mark(pl, pl->ev_sym, 7, st);
-    s = launch_symbolic_cta<1024>(pl, 7, st);
-    if (s != SPSYRK_OK) return s;
-    mark(pl, pl->ev_sym, 8, st);
-    SPSYRK_CUDA_TRY(cudaGetLastError());
-    SPSYRK_CUDA_TRY(exclusive_scan_i64<int32_t>(pl->cnt, rows, d_c_rowptr, pl->partials, st));
+    const int32_t* counts = pl->cnt;
+    if (pl->upper_active) {
+        spsyrk_plan_s* up = pl->upper;
+        up->map = with_map ? pl->map + pl->map_items : nullptr;  // the upper parts' words follow the lower parts'
+        up->map_bytes = with_map ? (size_t)up->map_items * sizeof(uint16_t) : 0;
+        s = symbolic_view(up, with_map, st);
+        if (s != SPSYRK_OK) return s;
+        if (rows > 0) {
+            add_counts_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(pl->cnt, up->cnt, rows, pl->cnt_tot);
+            note_launches(1);
+        }
+        counts = pl->cnt_tot;
+    }
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<int32_t>(counts, rows, d_c_rowptr, pl->partials, st));
+    if (pl->upper_active && rows > 0) {
+        // the upper part of row r starts after its lower part
+        upper_begin_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(d_c_rowptr, pl->cnt, rows, pl->hi_begin);
+        note_launches(1);
+    }
     int64_t nnz = 0;
     SPSYRK_CUDA_TRY(cudaMemcpyAsync(&nnz, d_c_rowptr + rows, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
     s = read_err(pl, st);
@@ -696,6 +827,7 @@ spsyrk_status_t spsyrk_symbolic(spsyrk_plan_t plan, int64_t* d_c_rowptr, int64_t
     *nnz_out = nnz;
     pl->have_symbolic = true;
     pl->map_filled = with_map;
+    if (pl->upper_active) { pl->upper->have_symbolic = true; pl->upper->map_filled = with_map; }
     return SPSYRK_OK;
 }
 
@@ -704,18 +836,30 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t* d_c_rowptr, in
     if (!plan || !d_c_rowptr) return SPSYRK_ERR_INVALID_ARG;
     spsyrk_plan_s* pl = plan;
     if (!pl->have_symbolic) return SPSYRK_ERR_SEQUENCE;
-    if (pl->work_total > 0 && (!d_c_colidx || !d_c_vals)) return SPSYRK_ERR_INVALID_ARG;
+    const int64_t work_all = pl->work_total + (pl->upper_active ? pl->upper->work_total : 0);
+    if (work_all > 0 && (!d_c_colidx || !d_c_vals)) return SPSYRK_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    switch (pl->dtype) {
-        case SPSYRK_F64: return numeric_typed<double>(pl, d_c_rowptr, d_c_colidx, d_c_vals, st);
-        case SPSYRK_F32: return numeric_typed<float>(pl, d_c_rowptr, d_c_colidx, d_c_vals, st);
-        default: return numeric_typed<int32_t>(pl, d_c_rowptr, d_c_colidx, d_c_vals, st);
-    }
+    auto run = [&](spsyrk_plan_s* v) {
+        switch (v->dtype) {
+            case SPSYRK_F64: return numeric_typed<double>(v, d_c_colidx, d_c_vals, st);
+            case SPSYRK_F32: return numeric_typed<float>(v, d_c_colidx, d_c_vals, st);
+            default: return numeric_typed<int32_t>(v, d_c_colidx, d_c_vals, st);
+        }
+    };
+    pl->out_begin = d_c_rowptr;
+    pl->out_end = pl->upper_active ? pl->hi_begin : d_c_rowptr + 1;
+    spsyrk_status_t s = run(pl);
+    if (s != SPSYRK_OK || !pl->upper_active) return s;
+    spsyrk_plan_s* up = pl->upper;
+    up->dev.jaccard = pl->dev.jaccard;
+    up->out_begin = pl->hi_begin;
+    up->out_end = d_c_rowptr + 1;
+    return run(up);
 }
 
 spsyrk_status_t spsyrk_plan_map_bytes(spsyrk_plan_t plan, size_t* bytes) {
     if (!plan || !bytes) return SPSYRK_ERR_INVALID_ARG;
-    *bytes = (size_t)plan->map_items * sizeof(uint16_t);
+    *bytes = (size_t)map_items_total(plan) * sizeof(uint16_t);
     return SPSYRK_OK;
 }
 
@@ -725,6 +869,7 @@ spsyrk_status_t spsyrk_plan_lend_map(spsyrk_plan_t plan, void* d_map, size_t byt
     plan->map_bytes = d_map ? bytes : 0;
     plan->map_filled = false;
     plan->have_symbolic = false;
+    if (plan->upper) { plan->upper->map_filled = false; plan->upper->have_symbolic = false; }
     return SPSYRK_OK;
 }
 
@@ -732,12 +877,13 @@ spsyrk_status_t spsyrk_plan_set_jaccard(spsyrk_plan_t plan, float* d_jaccard) {
     if (!plan) return SPSYRK_ERR_INVALID_ARG;
     if (d_jaccard && plan->dtype != SPSYRK_I32) return SPSYRK_ERR_INVALID_ARG;
     plan->dev.jaccard = d_jaccard;
+    if (plan->upper) plan->upper->dev.jaccard = d_jaccard;
     return SPSYRK_OK;
 }
 
 spsyrk_status_t spsyrk_plan_stats(spsyrk_plan_t plan, int64_t* work_total, int64_t class_rows[8]) {
     if (!plan) return SPSYRK_ERR_INVALID_ARG;
-    if (work_total) *work_total = plan->work_total;
+    if (work_total) *work_total = plan->work_total + (plan->upper_active ? plan->upper->work_total : 0);
     if (class_rows)
         for (int c = 0; c < NCLASS; ++c) class_rows[c] = plan->class_start[c + 1] - plan->class_start[c];
     return SPSYRK_OK;
@@ -749,7 +895,7 @@ spsyrk_status_t spsyrk_plan_buffers(spsyrk_plan_t plan, const int64_t** d_colptr
     if (d_colptr) *d_colptr = plan->dev.colptr;
     if (d_at_row) *d_at_row = plan->dev.at_row;
     if (d_at_val) *d_at_val = plan->dev.at_val;
-    if (d_work) *d_work = plan->dev.work;
+    if (d_work) *d_work = plan->upper_active ? plan->work_sum : plan->dev.work;
     return SPSYRK_OK;
 }
 
@@ -757,6 +903,7 @@ void spsyrk_destroy(spsyrk_plan_t plan) {
     if (!plan) return;
     if (plan->timing)
         for (int i = 0; i <= NCLASS; ++i) { cudaEventDestroy(plan->ev_sym[i]); cudaEventDestroy(plan->ev_num[i]); }
+    delete plan->upper;
     delete plan;
 }
 

@@ -39,7 +39,7 @@ template <typename V, int THREADS, bool NUMERIC, bool GLOBAL_ACC = false>
 __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int32_t* __restrict__ rows,
                                                            uint32_t chunk_bits, uint32_t acc_slots,
                                                            int32_t* __restrict__ cnt,
-                                                           const int64_t* __restrict__ c_rowptr,
+                                                           const int64_t* __restrict__ c_rowptr, const int64_t* __restrict__ c_rowend,
                                                            int32_t* __restrict__ c_colidx, V* __restrict__ c_vals,
                                                            uint32_t nrows = 0, uint32_t* row_counter = nullptr,
                                                            typename AccOf<V>::type* gscratch = nullptr, uint32_t gslots = 0) {
@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     const uint32_t U = P.mode == SPSYRK_TRIL ? (uint32_t)i + 1u : (uint32_t)P.m;
     if (NUMERIC) {
         // rows that overflow the shared-memory tile (and are not full) belong to the global variant
-        const int64_t row_cnt = c_rowptr[rloc + 1] - c_rowptr[rloc];
+        const int64_t row_cnt = c_rowend[rloc] - c_rowptr[rloc];
         const bool wants_global = gslots > 0 && row_cnt > (int64_t)acc_slots && U <= chunk_bits && row_cnt < (int64_t)U &&
                                   row_cnt <= (int64_t)gslots;
         if (wants_global != GLOBAL_ACC) return;
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     const int64_t p0 = P.rowptr[i];
     const uint32_t deg = (uint32_t)(P.rowptr[i + 1] - p0);
     const int64_t out_base = NUMERIC ? c_rowptr[rloc] : 0;
-    const int64_t out_end = NUMERIC ? c_rowptr[rloc + 1] : 0;  // bounds-checked build: no write at or past it
+    const int64_t out_end = NUMERIC ? c_rowend[rloc] : 0;  // bounds-checked build: no write at or past it
     (void)out_end;
     uint32_t total_cnt = 0;
 

@@ -100,7 +100,9 @@ struct NumericWarpSmem {
 template <typename V, int N, int G, typename Key, bool DIAG>
 __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N))
 numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows, const int64_t* __restrict__ c_rowptr,
-                    int32_t* __restrict__ c_colidx, V* __restrict__ c_vals) {
+                    const int64_t* __restrict__ c_rowend, int32_t* __restrict__ c_colidx, V* __restrict__ c_vals) {
+    // c_rowptr[r] / c_rowend[r]: where row r's part of the output starts and ends (c_rowend = c_rowptr + 1 unless the
+    // rows are written in two parts, see the full-output mode of the plan)
     using Acc = typename AccOf<V>::type;
     using Rec = ColRec<V>;
     using SM = NumericWarpSmem<V, N>;
@@ -327,7 +329,7 @@ numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows, con
         __syncwarp();
 #ifdef SPSYRK_CHECKED
         {
-            const int64_t room = h_n.z ? c_rowptr[h_n.x + 1] - ob_n : 0;  // the row's entries counted by the symbolic pass
+            const int64_t room = h_n.z ? c_rowend[h_n.x] - ob_n : 0;  // the row's entries counted by the symbolic pass
             if (!SPSYRK_IN_RANGE((int64_t)total <= room && total <= NP - 1, P.err)) total = 0;
         }
 #endif
@@ -349,6 +351,7 @@ numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows, con
         hB = hA; lB = lNew; hA = hNew;
     }
     cp_async_wait<0>();
+    (void)c_rowend;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -728,8 +731,8 @@ __host__ __device__ constexpr int numeric_map_warps(int n) { return n >= 512 ? 2
 template <typename V, int N, int G, bool DIAG>
 __global__ void __launch_bounds__(numeric_map_warps(N) * 32)
 numeric_map_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_t* __restrict__ itemoff, int64_t nrows,
-                        const uint16_t* __restrict__ map, const int64_t* __restrict__ c_rowptr, int32_t* __restrict__ c_colidx,
-                        V* __restrict__ c_vals) {
+                        const uint16_t* __restrict__ map, const int64_t* __restrict__ c_rowptr, const int64_t* __restrict__ c_rowend,
+                        int32_t* __restrict__ c_colidx, V* __restrict__ c_vals) {
     using Acc = typename AccOf<V>::type;
     using Rec = ColRec<V>;
     using SM = NumericMapSmem<V, N>;
@@ -829,7 +832,7 @@ numeric_map_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_t*
     Lists lB = load_lists(hB);
     int64_t ioB = n + stride < nrows ? itemoff[n + stride] : 0;
     uint4 h_n = h0;
-    int64_t ob_n = h0.z ? c_rowptr[h0.x] : 0, oe_n = h0.z ? c_rowptr[h0.x + 1] : 0;
+    int64_t ob_n = h0.z ? c_rowptr[h0.x] : 0, oe_n = h0.z ? c_rowend[h0.x] : 0;
     uint32_t w_n = issue(l0, n < nrows ? itemoff[n] : 0, 0);
     int b = 0;
 
@@ -837,7 +840,7 @@ numeric_map_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, const int64_t*
         const uint4 hNew = load_hdr(n + 3 * stride);
         const Lists lNew = load_lists(hA);
         const int64_t ioNew = n + 2 * stride < nrows ? itemoff[n + 2 * stride] : 0;
-        const int64_t ob_next = hB.z ? c_rowptr[hB.x] : 0, oe_next = hB.z ? c_rowptr[hB.x + 1] : 0;
+        const int64_t ob_next = hB.z ? c_rowptr[hB.x] : 0, oe_next = hB.z ? c_rowend[hB.x] : 0;
         const uint32_t w_next = issue(lB, ioB, b ^ 1);
 
         cp_async_wait<1>();
