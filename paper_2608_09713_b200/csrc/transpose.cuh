@@ -4,8 +4,9 @@
 //   colptr[n+1]        column pointers (int64)
 //   at_row[q], at_val[q]  entries of the column lists, q in [colptr[k], colptr[k+1]) ascending by row
 //   desc[p] = (start, len) for nonzero p = (i, k) of A: start = colptr[k]; len = number of entries
-//             of column k with row <= i (TRIL: the rank of i in the list, plus one) or the whole
-//             column length (FULL).  "Rows j <= i of column k" is then at_row[start, start+len).
+//             of column k with row <= i (the rank of i in the list, plus one).  "Rows j <= i of
+//             column k" is then at_row[start, start+len).  The full-output mode also keeps the rest of
+//             the list, the rows j > i, as a second descriptor (start + len, column length - len).
 //
 // Method: histogram of column ids and scan for colptr; then a stable LSD radix sort of the
 // nonzeros by column id with (row, value, position in A) as payload.  The nonzeros enter in row
@@ -172,13 +173,18 @@ static __global__ void __launch_bounds__(256) row_expand_kernel(const int64_t* _
 template <typename VB>
 struct EmitTransposeFinal {
     PlanDev P;
+    uint2* desc_hi;  // null in lower-triangle mode
     __device__ __forceinline__ void operator()(int64_t s, uint32_t k, uint32_t row, VB val, uint32_t p) const {
         const int64_t cs = P.colptr[k];
         P.at_row[s] = (int32_t)row;
         static_cast<VB*>(P.at_val)[s] = val;  // bit copy of the value that travelled with the element
         if constexpr (sizeof(VB) == 8) static_cast<uint4*>(P.at_rec)[s] = make_uint4(row, 0u, (uint32_t)val, (uint32_t)(val >> 32));
         else static_cast<uint2*>(P.at_rec)[s] = make_uint2(row, (uint32_t)val);
-        P.desc[p] = make_uint2((uint32_t)cs, P.mode == SPSYRK_TRIL ? (uint32_t)(s - cs) + 1u : (uint32_t)(P.colptr[k + 1] - cs));
+        // the entries of column k with row <= i are the first rank + 1 of its list; the full-output mode also keeps
+        // the rest of the list (rows > i) as a second descriptor
+        const uint32_t rank1 = (uint32_t)(s - cs) + 1u;
+        P.desc[p] = make_uint2((uint32_t)cs, rank1);
+        if (desc_hi) desc_hi[p] = make_uint2((uint32_t)cs + rank1, (uint32_t)(P.colptr[k + 1] - cs) - rank1);
     }
 };
 
@@ -186,7 +192,8 @@ struct EmitTransposeFinal {
 // a contiguous piece of its (row-sorted) list, so the descriptor of every nonzero of the rows
 // [r0, r1) is narrowed to that piece by two binary searches inside its full-range prefix.
 template <int G>
-static __global__ void __launch_bounds__(256) block_desc_kernel(PlanDev P, const uint2* __restrict__ desc_full,
+// desc_hi (full-output mode): the rest of every column list; the block is then cut out of the whole list.
+static __global__ void __launch_bounds__(256) block_desc_kernel(PlanDev P, const uint2* __restrict__ desc_full, const uint2* __restrict__ desc_hi,
                                                                 uint2* __restrict__ desc_blk, int32_t s0, int32_t s1) {
     const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
     const int gl = threadIdx.x & (G - 1);
@@ -194,7 +201,8 @@ static __global__ void __launch_bounds__(256) block_desc_kernel(PlanDev P, const
     const int64_t i = P.r0 + gid;
     const int64_t p0 = P.rowptr[i], p1 = P.rowptr[i + 1];
     for (int64_t p = p0 + gl; p < p1; p += G) {
-        const uint2 full = desc_full[p];
+        uint2 full = desc_full[p];
+        if (desc_hi) full.y += desc_hi[p].y;
         const int32_t* lst = P.at_row + full.x;
         const uint32_t lo = s0 <= 0 ? 0u : lower_bound_i32(lst, full.y, s0);
         const uint32_t hi = lower_bound_i32(lst, full.y, s1);
