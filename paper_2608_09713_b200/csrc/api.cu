@@ -122,11 +122,8 @@ size_t carve(spsyrk_plan_s* pl, spsyrk_plan_s* up, void* ws, int64_t m, int64_t 
     const int64_t items = std::max<int64_t>(std::max(m, n), 1);
     const int64_t nb = bin_blocks(items);
     auto colptr = c.take<int64_t>(n + 1);
-    auto at_row = c.take<int32_t>(nnz + 4);  // the symbolic gathers read aligned 16-byte pieces: up to 3 entries past the end
     auto at_val = c.take<char>(nnz * sv);
-    auto at_rec = c.take<char>(nnz * (sv == 8 ? 16 : 8));
     auto desc = c.take<uint2>(nnz);
-    auto desc_blk = c.take<uint2>(nnz);
     auto work = c.take<int64_t>(m);
     auto perm = c.take<int32_t>(m);
     auto hdr = c.take<uint4>(m);
@@ -134,14 +131,30 @@ size_t carve(spsyrk_plan_s* pl, spsyrk_plan_s* up, void* ws, int64_t m, int64_t 
     auto cls = c.take<uint8_t>(items);
     auto colcnt = c.take<uint32_t>(n);
     const int64_t rx_hist_n = (int64_t)(1 << TRANSPOSE_RADIX_BITS) * std::max<int64_t>(radix_tiles(nnz), 1);
-    auto rx_key_a = c.take<uint32_t>(nnz);
-    auto rx_row_a = c.take<uint32_t>(nnz);
-    auto rx_pos_a = c.take<uint32_t>(nnz);
-    auto rx_key_b = c.take<uint32_t>(nnz);
-    auto rx_row_b = c.take<uint32_t>(nnz);
-    auto rx_pos_b = c.take<uint32_t>(nnz);
-    auto rx_val_a = c.take<char>(nnz * sv);
-    auto rx_val_b = c.take<char>(nnz * sv);
+    // The two buffer sets of the radix sort (key, row, position, value per nonzero) are reused: the set that
+    // the last pass does not read receives the column lists that pass writes (row ids and records), and the
+    // set it does read holds, once the sort is over, the block descriptors and the heavy-row accumulator slices.
+    const uint32_t gslots = pow2_at_least((uint64_t)std::max<int64_t>(m, 1), 1024u, ROW_CHUNK_BITS_MAX_NUMERIC);
+    const size_t gacc_bytes = (size_t)GLOBAL_ACC_CTAS * gslots * sizeof(double);
+    const size_t set_bytes = std::max((size_t)nnz * (12 + sv) + 4 * ALIGN, (size_t)nnz * 8 + gacc_bytes + 2 * ALIGN);
+    auto set_a = c.take<char>(set_bytes);
+    auto set_b = c.take<char>(set_bytes);
+    Carver ca(set_a), cb(set_b);
+    auto rx_key_a = ca.take<uint32_t>(nnz);
+    auto rx_row_a = ca.take<uint32_t>(nnz);
+    auto rx_pos_a = ca.take<uint32_t>(nnz);
+    auto rx_val_a = ca.take<char>(nnz * sv);
+    auto rx_key_b = cb.take<uint32_t>(nnz);
+    auto rx_row_b = cb.take<uint32_t>(nnz);
+    auto rx_pos_b = cb.take<uint32_t>(nnz);
+    auto rx_val_b = cb.take<char>(nnz * sv);
+    const int npass = (bits_for((uint64_t)std::max<int64_t>(n - 1, 1)) + TRANSPOSE_RADIX_BITS - 1) / TRANSPOSE_RADIX_BITS;
+    const bool last_reads_a = npass >= 2 && (npass % 2) == 0;  // pass p writes set A when p is even; one pass reads the input itself (and row ids kept in set B)
+    Carver c_free(last_reads_a ? set_b : set_a), c_src(last_reads_a ? set_a : set_b);
+    auto at_row = c_free.take<int32_t>(nnz + 4);  // the symbolic gathers read aligned 16-byte pieces: up to 3 entries past the end
+    auto at_rec = c_free.take<char>(nnz * (sv == 8 ? 16 : 8));
+    auto desc_blk = c_src.take<uint2>(nnz);
+    auto gacc = c_src.take<double>((size_t)GLOBAL_ACC_CTAS * gslots);
     auto rx_hist = c.take<uint32_t>(rx_hist_n);
     auto rx_offsets = c.take<int64_t>(rx_hist_n + 1);
     auto blockhist = c.take<int32_t>(NCLASS * nb);
@@ -158,9 +171,6 @@ size_t carve(spsyrk_plan_s* pl, spsyrk_plan_s* up, void* ws, int64_t m, int64_t 
     auto facts = c.take<uint32_t>(64);  // [0..2] binary analysis, [32..63] its histogram
     auto adeg = c.take<int32_t>(std::max<int64_t>(m, 1));
     auto part_bounds = c.take<int64_t>(MAX_PARTS + 1);
-    // one global accumulator slice per persistent CTA of the heavy-row numeric kernel
-    const uint32_t gslots = pow2_at_least((uint64_t)std::max<int64_t>(m, 1), 1024u, ROW_CHUNK_BITS_MAX_NUMERIC);
-    auto gacc = c.take<double>((size_t)GLOBAL_ACC_CTAS * gslots);
     // full-output mode: the upper view's own per-row arrays and the second descriptor array
     uint2* desc_hi = nullptr;
     int64_t *u_work = nullptr, *u_itemoff = nullptr, *u_class_start_dev = nullptr, *hi_begin = nullptr, *work_sum = nullptr;
