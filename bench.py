@@ -34,7 +34,7 @@ METRIC = "tril_syrk_useful_multiply_adds_per_s"
 UNIT = "MAC/s"
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (bytes per useful multiply-add, multiplied by the launch's multiply-adds); None = not captured.
-NCU_TRAFFIC_BYTES_PER_MAC = 34.5
+NCU_TRAFFIC_BYTES_PER_MAC = 32.8
 
 
 def measured_peaks():
