@@ -38,5 +38,10 @@ def test_single_process_needs_no_process_group():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5
     assert bench.whole_job_rate(10.0, 1, 1000.0) == 10.0
-    w = bench.class_of_rows(torch.tensor([0, 10, 40, 600, 20000]).numpy(), torch.tensor([0, 3, 5, 40, 9]).numpy())
-    assert list(w) == [0, 1, 2, 6, 7]
+    work = torch.tensor([0, 10, 40, 600, 20000, 36]).numpy()
+    deg = torch.tensor([0, 3, 5, 40, 9, 5]).numpy()
+    w = bench.class_of_rows(work, deg, work)
+    assert list(w) == [0, 1, 2, 6, 7, 2]
+    # lower-triangle mode classes a light row by its products without the d_i diagonal ones
+    w = bench.class_of_rows(work - deg, deg, work)
+    assert list(w) == [0, 1, 2, 6, 7, 1]
