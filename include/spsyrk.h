@@ -172,6 +172,10 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t *d_c_rowptr,
  *   3. all pointers set: writes d_f_rowptr[m + 1] and fills d_f_colidx / d_f_vals (nnz_full entries).
  *      Asynchronous.  An entry above the diagonal that step 2 could not see (a row that is not
  *      ascending) is left out of the reflection; it never indexes outside the arrays.
+ *      Until this step's work on the stream has completed, d_f_colidx and d_f_vals (the sizes step 2
+ *      gave: nnz_full entries each) also serve as scratch of the sort, which is why the workspace is about
+ *      1.5 (8-byte values) to 2.2 (4-byte values) times the bytes of C_L and not 3 times; both arrays must
+ *      be 16-byte aligned and must not overlap each other, the workspace or C_L (INVALID_ARG if misaligned).
  * nnz_l = d_l_rowptr[m].  Errors: INVALID_ARG, WORKSPACE, BAD_CSR (an entry above the diagonal), CUDA.
  */
 spsyrk_status_t spsyrk_mirror(int64_t m, int64_t nnz_l, spsyrk_dtype_t dtype,

@@ -33,9 +33,10 @@ struct MirrorWs {
     uint32_t* rowtot;  // m
     int64_t* dcount;   // m + 1: diagonal entries of the rows before (exclusive prefix sums of diagf)
     int64_t* fbase;    // m: l_rowptr[j + 1] - dcount[j + 1]
-    // 8-byte values: two record buffers and two digit-byte buffers (nnz_l entries each)
-    MirrorRec *rec_a, *rec_b;
-    uint8_t *dig_a, *dig_b;
+    // 8-byte values: the record buffer the last pass reads (nnz_l records), the tail of the buffer that lives in
+    // F's value array, and digit bytes for inputs too small to keep them in F's column array
+    MirrorRec *rec_keep, *rec_tail;
+    uint8_t* dig_small;
     int32_t* tile_rows;  // 2 per tile
     unsigned long long* seg_start;  // m: first sorted position of column j's strictly lower entries
     unsigned long long* seg_end;    // m: one past the last
@@ -47,6 +48,16 @@ struct MirrorWs {
     uint32_t* hist;
     int64_t* offsets;
 };
+
+// Scratch inside the output.  Until the last pass writes it, F's memory is free, and the sort needs two record
+// buffers of 16 nnz_l bytes each.  The buffer the last pass reads must lie outside F; the other one lives in F's
+// value array, which holds 8 (2 nnz_l - D) bytes with D <= min(m, nnz_l) diagonal entries: the first
+// nnz_l - ceil(min(m, nnz_l) / 2) records always fit, the few remaining ones go to a tail in the workspace.
+// The digit bytes (two buffers of nnz_l bytes) live in F's column array (4 (2 nnz_l - D) bytes), which is free
+// whenever a histogram reads them: the last pass, the first to write that array, starts after its histogram.
+inline int mirror_passes_4byte(int64_t m) { return (bits_for((uint64_t)m) + MIRROR_RADIX_BITS - 1) / MIRROR_RADIX_BITS; }  // keys run from 0 to m
+inline int64_t mirror_tail_records(int64_t m, int64_t nnz_l) { return (std::min(m, nnz_l) + 1) / 2; }
+constexpr int64_t MIRROR_DIG_SMALL = 32;  // inputs of fewer entries than this keep their digit bytes in the workspace
 
 size_t carve(MirrorWs* w, void* ws, int64_t m, int64_t nnz_l, size_t sv) {
     char* base = static_cast<char*>(ws);
@@ -71,22 +82,28 @@ size_t carve(MirrorWs* w, void* ws, int64_t m, int64_t nnz_l, size_t sv) {
     t.err = (uint32_t*)take(8);  // [0] error word, [1] number of diagonal entries
     t.key_a = t.row_a = t.key_b = t.row_b = nullptr;
     t.val_a = t.val_b = nullptr;
-    t.rec_a = t.rec_b = nullptr;
-    t.dig_a = t.dig_b = nullptr;
+    t.rec_keep = t.rec_tail = nullptr;
+    t.dig_small = nullptr;
     t.tile_rows = nullptr;
     if (sv == 8) {
-        t.rec_a = (MirrorRec*)take(ne * sizeof(MirrorRec));
-        t.rec_b = (MirrorRec*)take(ne * sizeof(MirrorRec));
-        t.dig_a = (uint8_t*)take(ne);
-        t.dig_b = (uint8_t*)take(ne);
+        t.rec_keep = (MirrorRec*)take(ne * sizeof(MirrorRec));
+        t.rec_tail = (MirrorRec*)take((mirror_tail_records(m, nnz_l) + 1) * sizeof(MirrorRec));
+        t.dig_small = (uint8_t*)take(2 * MIRROR_DIG_SMALL);
         t.tile_rows = (int32_t*)take(2 * std::max<int64_t>(mirror_tiles(nnz_l), 1) * 4);
     } else {
-        t.key_a = (uint32_t*)take(ne * 4);
+        // The buffer set the last pass does not read keeps its keys in F's column array and its values in F's
+        // value array (4 (2 nnz_l - D) >= 4 nnz_l bytes each, free until the last pass); only its row ids need
+        // workspace.  Passes alternate A, B, A, ...: the last one reads B when the number of passes is odd.
+        const bool a_in_f = (mirror_passes_4byte(m) % 2) == 1;
         t.row_a = (uint32_t*)take(ne * 4);
-        t.key_b = (uint32_t*)take(ne * 4);
         t.row_b = (uint32_t*)take(ne * 4);
-        t.val_a = take(ne * sv);
-        t.val_b = take(ne * sv);
+        if (a_in_f) {
+            t.key_b = (uint32_t*)take(ne * 4);
+            t.val_b = take(ne * sv);
+        } else {
+            t.key_a = (uint32_t*)take(ne * 4);
+            t.val_a = take(ne * sv);
+        }
     }
     t.hist = (uint32_t*)take(hist_n * 4);
     t.offsets = (int64_t*)take((hist_n + 1) * 8);
@@ -240,9 +257,13 @@ int group_width(int64_t nnz, int64_t m) {
 }
 
 template <typename V>
-spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const int64_t* l_rowptr, const int32_t* l_colidx,
+spsyrk_status_t mirror_fill(const MirrorWs& ws, int64_t m, int64_t nnz_l, const int64_t* l_rowptr, const int32_t* l_colidx,
                             const void* l_vals, int64_t* f_rowptr, int32_t* f_colidx, void* f_vals, cudaStream_t st) {
     constexpr int BITS = MIRROR_RADIX_BITS;
+    MirrorWs w = ws;
+    // the buffer set without keys and values of its own keeps them in F's arrays (see carve)
+    if (!w.key_a) { w.key_a = reinterpret_cast<uint32_t*>(f_colidx); w.val_a = f_vals; }
+    if (!w.key_b) { w.key_b = reinterpret_cast<uint32_t*>(f_colidx); w.val_b = f_vals; }
     const V* lv = static_cast<const V*>(l_vals);
     V* fv = static_cast<V*>(f_vals);
     const int g = group_width(nnz_l, m);
@@ -260,7 +281,7 @@ spsyrk_status_t mirror_fill(const MirrorWs& w, int64_t m, int64_t nnz_l, const i
         }
 #undef EXPAND
         note_launches(1);
-        const int npass = (bits_for((uint64_t)m) + BITS - 1) / BITS;  // keys run from 0 to m
+        const int npass = mirror_passes_4byte(m);
         const uint32_t* src_key = w.key_b;
         const uint32_t* src_row = w.row_b;
         const V* src_val = lv;
@@ -363,6 +384,8 @@ spsyrk_status_t mirror_fill_rec(const MirrorWs& w, int64_t m, int64_t nnz_l, con
     const uint64_t* lv = static_cast<const uint64_t*>(l_vals);
     uint64_t* fv = static_cast<uint64_t*>(f_vals);
     const int g = group_width(nnz_l, m);
+    // F's arrays hold records and digit bytes during the sort: both must take 16-byte accesses
+    if (nnz_l > 0 && ((reinterpret_cast<uintptr_t>(f_vals) | reinterpret_cast<uintptr_t>(f_colidx)) & 15u)) return SPSYRK_ERR_INVALID_ARG;
     if (m > 0) {
         SPSYRK_CUDA_TRY(cudaMemsetAsync(w.seg_start, 0xff, (size_t)m * 8, st));
         SPSYRK_CUDA_TRY(cudaMemsetAsync(w.seg_end, 0, (size_t)m * 8, st));
@@ -382,18 +405,29 @@ spsyrk_status_t mirror_fill_rec(const MirrorWs& w, int64_t m, int64_t nnz_l, con
         a.fbase = w.fbase; a.f_colidx = f_colidx; a.f_vals = fv; a.seg_start = w.seg_start; a.seg_end = w.seg_end;
         a.dtotal = w.dcount + m; a.err = w.err;
         g_mirror_passes = 0;
+        // buffers: pass p writes records X[p] and digits Y[p]; X[npass - 2] is the one the last pass reads
+        MirrorRec* const alias = reinterpret_cast<MirrorRec*>(fv);
+        const int64_t alias_split = nnz_l - mirror_tail_records(m, nnz_l);
+        const int64_t dig_stride = (nnz_l + 15) / 16 * 16;
+        uint8_t* const dig0 = nnz_l < MIRROR_DIG_SMALL ? w.dig_small : reinterpret_cast<uint8_t*>(f_colidx);
+        uint8_t* const dig1 = nnz_l < MIRROR_DIG_SMALL ? w.dig_small + MIRROR_DIG_SMALL : dig0 + dig_stride;
+        auto in_keep = [&](int p) { return ((npass - 2 - p) % 2) == 0; };  // does pass p write the workspace buffer?
         for (int p = 0; p < npass; ++p) {
             const bool first = p == 0, last = p == npass - 1;
-            const bool to_a = (p % 2) == 0;
             if (g_mirror_timing && p < MIRROR_MAX_PASSES) cudaEventRecord(g_mirror_ev[p], st);
             const unsigned hb = (unsigned)((nt + MR_HIST_TILES - 1) / MR_HIST_TILES);
             if (first) mirror_hist_key_kernel<BITS><<<hb, MR_THREADS, 0, st>>>(reinterpret_cast<const uint32_t*>(l_colidx), nnz_l, 0, w.hist, nt);
-            else radix_hist_u8_kernel<BITS><<<hb, MR_THREADS, 0, st>>>(to_a ? w.dig_b : w.dig_a, nnz_l, w.hist, nt);
+            else radix_hist_u8_kernel<BITS><<<hb, MR_THREADS, 0, st>>>(((p - 1) % 2) == 0 ? dig0 : dig1, nnz_l, w.hist, nt);
             note_launches(1);
             SPSYRK_CUDA_TRY(exclusive_scan_i64<uint32_t>(w.hist, (int64_t)NB * nt, w.offsets, w.partials, st));
-            a.src = to_a ? w.rec_b : w.rec_a;
-            a.dst = to_a ? w.rec_a : w.rec_b;
-            a.next_digit = to_a ? w.dig_a : w.dig_b;
+            const bool src_keep = !first && in_keep(p - 1), dst_keep = in_keep(p);
+            a.src = src_keep ? w.rec_keep : alias;
+            a.src_tail = w.rec_tail;
+            a.src_split = src_keep ? nnz_l : alias_split;
+            a.dst = dst_keep ? w.rec_keep : alias;
+            a.dst_tail = w.rec_tail;
+            a.dst_split = dst_keep ? nnz_l : alias_split;
+            a.next_digit = (p % 2) == 0 ? dig0 : dig1;
             cudaError_t e;
             if (first && last) e = launch_mirror_pass<true, true>(a, nnz_l, p * BITS, w.offsets, nt, st);
             else if (first) e = launch_mirror_pass<true, false>(a, nnz_l, p * BITS, w.offsets, nt, st);

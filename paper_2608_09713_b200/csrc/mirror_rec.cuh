@@ -128,9 +128,15 @@ struct MirrorPassArgs {
     const uint64_t* l_vals;
     int64_t m;
     const int32_t* tile_rows;  // [2 * tiles]: row of each tile's first and last entry
+    // A record buffer comes in two pieces: records [0, split) at `src` / `dst`, the rest at the tail pointer.
+    // (The buffer that lives in F's value array while F is not yet written is a few records short; see mirror.cu.)
     const MirrorRec* src;
+    const MirrorRec* src_tail;
+    int64_t src_split;
     // destination: records and the next digit, or F (last pass)
     MirrorRec* dst;
+    MirrorRec* dst_tail;
+    int64_t dst_split;
     uint8_t* next_digit;
     const int64_t* fbase;  // l_rowptr[j + 1] - diagonals of rows 0..j
     int32_t* f_colidx;
@@ -215,7 +221,10 @@ __global__ void __launch_bounds__(MR_THREADS, MR_MIN_CTAS) mirror_pass_kernel(Mi
         for (int i = 0; i < MR_ITEMS; ++i) {
             const int t = warp * MR_CHUNK + i * 32 + lane;
             uint4 r = make_uint4(0u, 0u, 0u, 0u);
-            if (t < tile_n) r = reinterpret_cast<const uint4*>(A.src)[tile_base + t];  // one 16-byte load
+            if (t < tile_n) {  // one 16-byte load
+                const int64_t e = tile_base + t;
+                r = e < A.src_split ? reinterpret_cast<const uint4*>(A.src)[e] : reinterpret_cast<const uint4*>(A.src_tail)[e - A.src_split];
+            }
             k[i] = r.x; a[i] = r.y; b[i] = (uint64_t)r.z | ((uint64_t)r.w << 32);
         }
     }
@@ -297,7 +306,8 @@ __global__ void __launch_bounds__(MR_THREADS, MR_MIN_CTAS) mirror_pass_kernel(Mi
         const int64_t dest = goff[(r.key >> shift) & (NB - 1)] + q;
         if (!SPSYRK_IN_RANGE(dest >= 0 && dest < n, A.err)) continue;
         if (!FINAL) {
-            reinterpret_cast<uint4*>(A.dst)[dest] = r4;
+            if (dest < A.dst_split) reinterpret_cast<uint4*>(A.dst)[dest] = r4;
+            else reinterpret_cast<uint4*>(A.dst_tail)[dest - A.dst_split] = r4;
             A.next_digit[dest] = (uint8_t)((r.key >> (shift + BITS)) & (NB - 1));
         } else if (r.key < (uint32_t)A.m) {
             // ends of a run of one key inside the tile; a segment that spans tiles settles through min / max

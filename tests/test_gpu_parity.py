@@ -217,10 +217,11 @@ def test_mirror_rejects_upper_entries(B):
 
 
 @pytest.mark.parametrize("m,density,diag", [(7, 0.5, "some"), (200, 0.1, "some"), (200, 0.1, "none"), (3000, 0.004, "all"),
-                                            (70000, 0.0001, "some")])
+                                            (70000, 0.0001, "some"), (2 ** 24 + 77, 2e-8, "some")])
 def test_mirror_general_lower_triangles(B, m, density, diag):
     """Lower triangles that are not products: rows without a diagonal entry, empty rows, one pass
-    (m < 256) up to three radix passes (m > 65536)."""
+    (m < 256) up to four radix passes (m > 2^24); with every diagonal stored the record buffer that
+    lives in F's value array is at its shortest."""
     rng = np.random.default_rng(m)
     nnz_target = int(density * m * m / 2) + m
     r = rng.integers(0, m, size=nnz_target)
@@ -234,9 +235,23 @@ def test_mirror_general_lower_triangles(B, m, density, diag):
     r, c = key // m, key % m
     rp = np.zeros(m + 1, dtype=np.int64)
     np.cumsum(np.bincount(r, minlength=m), out=rp[1:])
-    vals = rng.standard_normal(c.size)
-    got = B.spsyrk_mirror(m, torch.from_numpy(rp).cuda(), torch.from_numpy(c.astype(np.int32)).cuda(), torch.from_numpy(vals).cuda())
-    exp = oracle.mirror(m, rp, c.astype(np.int32), vals)
+    for dtype in (np.float64, np.float32):      # 16-byte records / separate arrays: both keep scratch in F's arrays
+        vals = rng.standard_normal(c.size).astype(dtype)
+        got = B.spsyrk_mirror(m, torch.from_numpy(rp).cuda(), torch.from_numpy(c.astype(np.int32)).cuda(), torch.from_numpy(vals).cuda())
+        exp = oracle.mirror(m, rp, c.astype(np.int32), vals.astype(np.float64))
+        assert np.array_equal(got[0].cpu().numpy(), exp[0]) and np.array_equal(got[1].cpu().numpy(), exp[1])
+        assert np.array_equal(got[2].cpu().numpy().astype(np.float64), exp[2])
+
+
+def test_mirror_few_entries_many_rows(B):
+    """Three radix passes over five entries: the digit bytes do not fit F's column array and stay in the workspace."""
+    m = 100000
+    r = np.array([5, 70000, 70000, 99999, 99999]); c = np.array([5, 5, 69999, 0, 99999], dtype=np.int32)
+    rp = np.zeros(m + 1, dtype=np.int64)
+    np.cumsum(np.bincount(r, minlength=m), out=rp[1:])
+    vals = np.arange(1.0, 6.0)
+    got = B.spsyrk_mirror(m, torch.from_numpy(rp).cuda(), torch.from_numpy(c).cuda(), torch.from_numpy(vals).cuda())
+    exp = oracle.mirror(m, rp, c, vals)
     for g, e in zip(got, exp):
         assert np.array_equal(g.cpu().numpy(), e)
 
