@@ -70,7 +70,7 @@ size_t carve(MirrorWs* w, void* ws, int64_t m, int64_t nnz_l, size_t sv) {
     };
     const int64_t items = std::max<int64_t>(m, 1);
     const int64_t ne = std::max<int64_t>(nnz_l, 1);
-    const int64_t hist_n = (int64_t)(1 << MIRROR_RADIX_BITS) * std::max<int64_t>(std::max(radix_tiles(nnz_l), mirror_tiles(nnz_l)), 1);
+    const int64_t hist_n = (int64_t)(1 << MIRROR_RADIX_BITS) * std::max<int64_t>(sv == 8 ? mirror_groups(nnz_l) : radix_tiles(nnz_l), 1);
     MirrorWs t;
     t.diagf = (uint32_t*)take(items * 4);
     t.rowtot = (uint32_t*)take(items * 4);
@@ -397,8 +397,9 @@ spsyrk_status_t mirror_fill_rec(const MirrorWs& w, int64_t m, int64_t nnz_l, con
         mirror_fbase_kernel<<<(unsigned)((m + 255) / 256), 256, 0, st>>>(l_rowptr, w.dcount, m, w.fbase);
         note_launches(1);
         const int npass = (bits_for((uint64_t)(m - 1 > 0 ? m - 1 : 1)) + BITS - 1) / BITS;  // keys are column ids below m
-        const int64_t nt = mirror_tiles(nnz_l);
-        mirror_tile_rows_kernel<<<(unsigned)((2 * nt + 255) / 256), 256, 0, st>>>(l_rowptr, m, nnz_l, nt, w.tile_rows);
+        const int64_t nt = mirror_groups(nnz_l);  // histogram columns and CTAs of a pass
+        const int64_t ntr = mirror_tiles(nnz_l);
+        mirror_tile_rows_kernel<<<(unsigned)((2 * ntr + 255) / 256), 256, 0, st>>>(l_rowptr, m, nnz_l, ntr, w.tile_rows);
         note_launches(1);
         MirrorPassArgs a{};
         a.l_rowptr = l_rowptr; a.l_colidx = l_colidx; a.l_vals = lv; a.m = m; a.tile_rows = w.tile_rows;
