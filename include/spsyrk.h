@@ -156,6 +156,19 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t *d_c_rowptr,
                                int32_t *d_c_colidx, void *d_c_vals, void *cuda_stream);
 
 /*
+ * spsyrk_numeric_rows - spsyrk_numeric for the output rows [row_begin, row_end) only (global row ids inside
+ * the plan's range).  The entries of these rows are written at the offsets d_c_rowptr gives them, exactly as
+ * spsyrk_numeric would; the rest of d_c_colidx / d_c_vals is not touched.  Calling it over a partition of the
+ * range therefore fills C_L block by block, e.g. to copy finished row blocks to the host while later ones are
+ * computed (row blocks are independent: Algorithm 2 works on any row range, the halving of the rows costs
+ * nothing).  Reads the positions of the range in the plan's row lists back (one stream synchronisation)
+ * before it launches.  Errors: INVALID_ARG (range outside the plan's), SEQUENCE, CUDA.
+ */
+spsyrk_status_t spsyrk_numeric_rows(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end,
+                                    const int64_t *d_c_rowptr, int32_t *d_c_colidx, void *d_c_vals,
+                                    void *cuda_stream);
+
+/*
  * spsyrk_mirror - materialise F = C_L + C_L^T - D, the full symmetric matrix, from a complete
  * (untiled or re-assembled) lower triangle (Section III-A: the full matrix, when it is needed, is
  * obtained from the stored half by a transpose; Section V-F: C = C_L + C_L^T - D).  Row i of F is row i of C_L followed by (r, c_ri) for
@@ -385,7 +398,10 @@ const char *spsyrk_status_string(spsyrk_status_t s);
  *   1. h_c_colidx == NULL: runs plan + symbolic, writes h_c_rowptr[m+1] and *nnz_out, keeps the
  *      device state in *session.
  *   2. with h_c_colidx / h_c_vals of *nnz_out entries: runs numeric, copies the result back and
- *      frees the session.
+ *      frees the session.  A large result is computed in up to eight row blocks of about equal
+ *      numbers of entries (spsyrk_numeric_rows) and each block is copied on a second stream while
+ *      the following ones are computed, so only the first block's computation is not hidden
+ *      behind the download.
  * Device memory for this entry point is allocated by the library (cudaMalloc) and kept in two
  * grow-only blocks per device between calls, because allocating and freeing several GB per call
  * costs more than the computation; spsyrk_host_release_cache frees the blocks of the current

@@ -47,6 +47,8 @@ _lib.spsyrk_plan_map_bytes.restype = _int
 _lib.spsyrk_plan_lend_map.argtypes = [_vp, _vp, ctypes.c_size_t]
 _lib.spsyrk_plan_lend_map.restype = _int
 _lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
+_lib.spsyrk_numeric_rows.argtypes = [_vp, _i64, _i64, _vp, _vp, _vp, _vp]
+_lib.spsyrk_numeric_rows.restype = _int
 _lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_column_panel.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_accumulate.argtypes = [_i64, _int, _i64, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
@@ -215,6 +217,13 @@ def spsyrk_numeric(plan: Plan, c_rowptr, c_colidx, c_vals, stream=None):
     _dev_check(c_rowptr, c_colidx, c_vals)
     assert c_colidx.dtype == torch.int32 and c_vals.dtype == plan.dtype
     _check(_lib.spsyrk_numeric(plan._h, _p(c_rowptr), _p(c_colidx), _p(c_vals), _stream(stream)), "spsyrk_numeric")
+
+
+def spsyrk_numeric_rows(plan: Plan, row_begin: int, row_end: int, c_rowptr, c_colidx, c_vals, stream=None):
+    _dev_check(c_rowptr, c_colidx, c_vals)
+    assert c_colidx.dtype == torch.int32 and c_vals.dtype == plan.dtype
+    _check(_lib.spsyrk_numeric_rows(plan._h, int(row_begin), int(row_end), _p(c_rowptr), _p(c_colidx), _p(c_vals), _stream(stream)),
+           "spsyrk_numeric_rows")
 
 
 def spsyrk_destroy(plan: Plan):

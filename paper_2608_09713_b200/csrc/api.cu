@@ -2,7 +2,9 @@
 // Host-side orchestration only; every step of the path runs in the kernels of the .cuh files.
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <new>
+#include <vector>
 
 #include "rows_cta.cuh"
 #include "rows_warp.cuh"
@@ -68,6 +70,10 @@ struct spsyrk_plan_s {
     int64_t* work_sum;      // rows: work of both parts
     const int64_t* out_begin;  // set by spsyrk_numeric: where each row's part starts / ends in the output
     const int64_t* out_end;
+    // spsyrk_numeric_rows: the numeric launches take only positions [sub_lo[c], sub_hi[c]) of class c's row list
+    bool sub_active;
+    int64_t sub_lo[NCLASS], sub_hi[NCLASS];
+    int64_t* host_pos;  // pinned, device-visible host memory the position search of spsyrk_numeric_rows writes into (4 * NCLASS)
     int64_t rows_cap;
     // workspace views
     int32_t* perm;
@@ -414,9 +420,15 @@ spsyrk_status_t launch_symbolic_warp(spsyrk_plan_s* pl, int c, cudaStream_t st) 
     return pl->diag ? launch_symbolic_warp_d<N, true>(pl, c, st) : launch_symbolic_warp_d<N, false>(pl, c, st);
 }
 
+// the part of class c's row list (rows in ascending order) a numeric launch covers
+inline int64_t numeric_first(const spsyrk_plan_s* pl, int c) { return pl->sub_active ? pl->sub_lo[c] : pl->class_start[c]; }
+inline int64_t numeric_count(const spsyrk_plan_s* pl, int c) {
+    return pl->sub_active ? pl->sub_hi[c] - pl->sub_lo[c] : pl->class_start[c + 1] - pl->class_start[c];
+}
+
 template <typename V, int N, typename Key, bool DIAG>
 spsyrk_status_t launch_numeric_warp_d(spsyrk_plan_s* pl, int c, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
-    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    const int64_t count = numeric_count(pl, c);
     if (count <= 0) return SPSYRK_OK;
     constexpr int G = warp_class_group(N);
     constexpr int NW = numeric_warps(N);
@@ -430,7 +442,7 @@ spsyrk_status_t launch_numeric_warp_d(spsyrk_plan_s* pl, int c, int32_t* c_colid
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
     const int64_t want = (count + ROWS - 1) / ROWS;
     const int64_t cap = (int64_t)pl->sm_count * per_sm;
-    kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], count, pl->out_begin, pl->out_end,
+    kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + numeric_first(pl, c), count, pl->out_begin, pl->out_end,
                                                                c_colidx, static_cast<V*>(c_vals));
     note_launches(1);
     return SPSYRK_OK;
@@ -471,7 +483,7 @@ spsyrk_status_t launch_symbolic_sort(spsyrk_plan_s* pl, int c, cudaStream_t st) 
 
 template <typename V, int N, bool DIAG>
 spsyrk_status_t launch_numeric_map_d(spsyrk_plan_s* pl, int c, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
-    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    const int64_t count = numeric_count(pl, c);
     if (count <= 0) return SPSYRK_OK;
     constexpr int G = warp_class_group(N);
     constexpr int NW = numeric_map_warps(N);
@@ -483,7 +495,7 @@ spsyrk_status_t launch_numeric_map_d(spsyrk_plan_s* pl, int c, int32_t* c_colidx
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, NW * 32, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
     const int64_t want = (count + ROWS - 1) / ROWS;
     const int64_t cap = (int64_t)pl->sm_count * per_sm;
-    kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + pl->class_start[c], pl->itemoff + pl->class_start[c],
+    kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + numeric_first(pl, c), pl->itemoff + numeric_first(pl, c),
                                                                count, pl->map, pl->out_begin, pl->out_end, c_colidx, static_cast<V*>(c_vals));
     note_launches(1);
     return SPSYRK_OK;
@@ -566,8 +578,9 @@ spsyrk_status_t launch_symbolic_cta(spsyrk_plan_s* pl, int c, cudaStream_t st) {
 template <typename V, int THREADS>
 spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_or_zero, int32_t* c_colidx, void* c_vals, cudaStream_t st) {
     using Acc = typename AccOf<V>::type;
-    const int64_t count = pl->class_start[c + 1] - pl->class_start[c];
+    const int64_t count = numeric_count(pl, c);
     if (count <= 0) return SPSYRK_OK;
+    const int32_t* rows_of_class = pl->perm + numeric_first(pl, c);
     const uint32_t cb = row_chunk_bits(pl, ROW_CHUNK_BITS_MAX_NUMERIC);
     uint32_t slots = acc_slots_or_zero;
     if (slots == 0) {
@@ -581,7 +594,7 @@ spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_
     // rows that overflow the shared-memory tile go to the persistent variant with global accumulators
     const bool use_global = acc_slots_or_zero == 0 && pl->gslots >= cb;
     const uint32_t gslots = use_global ? pl->gslots : 0u;
-    kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, pl->out_begin, pl->out_end,
+    kern<<<(unsigned)count, THREADS, smem, st>>>(pl->dev, rows_of_class, cb, slots, nullptr, pl->out_begin, pl->out_end,
                                                   c_colidx, static_cast<V*>(c_vals), 0u, nullptr, nullptr, gslots);
     note_launches(1);
     if (use_global) {
@@ -590,7 +603,7 @@ spsyrk_status_t launch_numeric_cta(spsyrk_plan_s* pl, int c, uint32_t acc_slots_
         SPSYRK_CUDA_TRY(cudaFuncSetAttribute(gkern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gsmem));
         SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->row_counter, 0, sizeof(uint32_t), st));
         const unsigned grid = (unsigned)std::min<int64_t>(std::min<int64_t>(pl->sm_count, GLOBAL_ACC_CTAS), count);
-        gkern<<<grid, THREADS, gsmem, st>>>(pl->dev, pl->perm + pl->class_start[c], cb, slots, nullptr, pl->out_begin, pl->out_end,
+        gkern<<<grid, THREADS, gsmem, st>>>(pl->dev, rows_of_class, cb, slots, nullptr, pl->out_begin, pl->out_end,
                                             c_colidx, static_cast<V*>(c_vals), (uint32_t)count, pl->row_counter,
                                             reinterpret_cast<Acc*>(pl->gacc), gslots);
         note_launches(1);
@@ -867,6 +880,78 @@ spsyrk_status_t spsyrk_numeric(spsyrk_plan_t plan, const int64_t* d_c_rowptr, in
     return run(up);
 }
 
+namespace {
+// Pinned host blocks for the read-back of spsyrk_numeric_rows.  Allocating pinned memory takes a millisecond or
+// more, so blocks of destroyed plans are kept for the next plan (a few hundred bytes each, never freed).
+std::mutex g_host_pos_mutex;
+std::vector<int64_t*> g_host_pos_pool;
+cudaError_t host_pos_acquire(int64_t** out) {
+    {
+        std::lock_guard<std::mutex> lock(g_host_pos_mutex);
+        if (!g_host_pos_pool.empty()) {
+            *out = g_host_pos_pool.back();
+            g_host_pos_pool.pop_back();
+            return cudaSuccess;
+        }
+    }
+    return cudaHostAlloc(reinterpret_cast<void**>(out), 4 * NCLASS * sizeof(int64_t), cudaHostAllocMapped | cudaHostAllocPortable);
+}
+void host_pos_release(int64_t* p) {
+    std::lock_guard<std::mutex> lock(g_host_pos_mutex);
+    g_host_pos_pool.push_back(p);
+}
+
+// out[(2 * c) + e] = first position of class c's row list (ascending local row ids) whose row is >= bound[e]
+__global__ void class_positions_kernel(const int32_t* __restrict__ perm, const int64_t* __restrict__ class_start_dev, int64_t lo_row,
+                                       int64_t hi_row, int64_t* __restrict__ out) {
+    const int t = threadIdx.x;
+    if (t >= 2 * NCLASS) return;
+    const int c = t >> 1;
+    const int64_t bound = (t & 1) ? hi_row : lo_row;
+    int64_t lo = class_start_dev[c], hi = class_start_dev[c + 1];
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((int64_t)perm[mid] < bound) lo = mid + 1; else hi = mid;
+    }
+    out[t] = lo;
+}
+}  // namespace
+
+spsyrk_status_t spsyrk_numeric_rows(spsyrk_plan_t plan, int64_t row_begin, int64_t row_end, const int64_t* d_c_rowptr,
+                                    int32_t* d_c_colidx, void* d_c_vals, void* cuda_stream) {
+    if (!plan || !d_c_rowptr) return SPSYRK_ERR_INVALID_ARG;
+    spsyrk_plan_s* pl = plan;
+    if (!pl->have_symbolic) return SPSYRK_ERR_SEQUENCE;
+    if (row_begin < pl->dev.r0 || row_end > pl->dev.r1 || row_begin > row_end) return SPSYRK_ERR_INVALID_ARG;
+    if (row_begin == row_end) return SPSYRK_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // where the rows of the range sit in every class's list: one small kernel per view and one read-back
+    // The kernel writes straight into pinned host memory: a device-to-host copy would queue behind whatever the
+    // caller is downloading at the moment (the point of this call is to overlap with such copies).
+    if (!pl->host_pos) SPSYRK_CUDA_TRY(host_pos_acquire(&pl->host_pos));
+    int64_t* dev_pos = nullptr;
+    SPSYRK_CUDA_TRY(cudaHostGetDevicePointer(reinterpret_cast<void**>(&dev_pos), pl->host_pos, 0));
+    spsyrk_plan_s* views[2] = {pl, pl->upper_active ? pl->upper : nullptr};
+    for (int v = 0; v < 2; ++v) {
+        if (!views[v]) continue;
+        class_positions_kernel<<<1, 32, 0, st>>>(views[v]->perm, views[v]->class_start_dev, row_begin - pl->dev.r0, row_end - pl->dev.r0,
+                                                 dev_pos + v * 2 * NCLASS);
+        note_launches(1);
+    }
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    SPSYRK_CUDA_TRY(cudaStreamSynchronize(st));
+    const int64_t(*pos)[2 * NCLASS] = reinterpret_cast<const int64_t(*)[2 * NCLASS]>(pl->host_pos);
+    for (int v = 0; v < 2; ++v) {
+        if (!views[v]) continue;
+        views[v]->sub_active = true;
+        for (int c = 0; c < NCLASS; ++c) { views[v]->sub_lo[c] = pos[v][2 * c]; views[v]->sub_hi[c] = pos[v][2 * c + 1]; }
+    }
+    const spsyrk_status_t s = spsyrk_numeric(plan, d_c_rowptr, d_c_colidx, d_c_vals, cuda_stream);
+    for (int v = 0; v < 2; ++v)
+        if (views[v]) views[v]->sub_active = false;
+    return s;
+}
+
 spsyrk_status_t spsyrk_plan_map_bytes(spsyrk_plan_t plan, size_t* bytes) {
     if (!plan || !bytes) return SPSYRK_ERR_INVALID_ARG;
     *bytes = (size_t)map_items_total(plan) * sizeof(uint16_t);
@@ -913,6 +998,7 @@ void spsyrk_destroy(spsyrk_plan_t plan) {
     if (!plan) return;
     if (plan->timing)
         for (int i = 0; i <= NCLASS; ++i) { cudaEventDestroy(plan->ev_sym[i]); cudaEventDestroy(plan->ev_num[i]); }
+    if (plan->host_pos) host_pos_release(plan->host_pos);
     delete plan->upper;
     delete plan;
 }

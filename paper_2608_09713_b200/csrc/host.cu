@@ -1,5 +1,6 @@
 // spsyrk_host_tril: the whole path on host buffers.  Device memory is allocated here with
 // cudaMalloc; the computation itself goes through the same entry points a device caller uses.
+#include <algorithm>
 #include <mutex>
 #include <new>
 
@@ -21,6 +22,8 @@ std::mutex g_arena_mutex;
 Arena g_arena[MAX_DEVICES][2];  // [device][0: inputs, workspace, row pointers; 1: output entries]
 
 constexpr size_t A256 = 256;
+constexpr int HOST_MAX_BLOCKS = 8;
+constexpr int64_t HOST_BLOCK_MIN_ENTRIES = int64_t(1) << 22;  // below this a block's launches cost more than its copy hides
 size_t up256(size_t b) { return (b + A256 - 1) / A256 * A256; }
 }  // namespace
 
@@ -34,6 +37,12 @@ struct spsyrk_session_s {
     bool cached[2] = {false, false};      // block i belongs to the device's arena (else: owned, freed on release)
     void *d_rowptr = nullptr, *d_colidx = nullptr, *d_vals = nullptr, *d_ws = nullptr;
     void *d_c_rowptr = nullptr, *d_c_colidx = nullptr, *d_c_vals = nullptr;
+    // call 2 computes and downloads C_L in row blocks of about equal numbers of entries: the copy of a block
+    // runs while the next ones are computed
+    cudaStream_t copy_stream = nullptr;
+    int blocks = 0;
+    int64_t block_row[HOST_MAX_BLOCKS + 1] = {};
+    int64_t block_off[HOST_MAX_BLOCKS + 1] = {};
 };
 
 namespace {
@@ -64,6 +73,10 @@ cudaError_t acquire(spsyrk_session_s* s, int which, size_t bytes) {
 void release(spsyrk_session_s* s) {
     if (!s) return;
     if (s->plan) spsyrk_destroy(s->plan);
+    if (s->copy_stream) {
+        cudaStreamSynchronize(s->copy_stream);
+        cudaStreamDestroy(s->copy_stream);
+    }
     if (s->stream) {
         cudaStreamSynchronize(s->stream);
         cudaStreamDestroy(s->stream);
@@ -134,6 +147,14 @@ extern "C" spsyrk_status_t spsyrk_host_tril(spsyrk_session_t* session, int64_t m
         HOST_ST(spsyrk_symbolic(s->plan, (int64_t*)s->d_c_rowptr, &s->nnz_c, s->stream));
         HOST_TRY(cudaMemcpyAsync(h_c_rowptr, s->d_c_rowptr, (size_t)(m + 1) * 8, cudaMemcpyDeviceToHost, s->stream));
         HOST_TRY(cudaStreamSynchronize(s->stream));
+        // row blocks of call 2: boundaries where the output reaches k / blocks of its entries
+        s->blocks = (int)std::max<int64_t>(1, std::min<int64_t>(HOST_MAX_BLOCKS, s->nnz_c / HOST_BLOCK_MIN_ENTRIES));
+        for (int b = 0; b <= s->blocks; ++b) {
+            const int64_t target = b == s->blocks ? s->nnz_c : s->nnz_c / s->blocks * b;
+            const int64_t r = b == s->blocks ? m : b == 0 ? 0 : std::lower_bound(h_c_rowptr, h_c_rowptr + m + 1, target) - h_c_rowptr;
+            s->block_row[b] = std::min<int64_t>(r, m);
+            s->block_off[b] = h_c_rowptr[s->block_row[b]];
+        }
         *nnz_out = s->nnz_c;
         *session = s;
         return SPSYRK_OK;
@@ -146,12 +167,35 @@ extern "C" spsyrk_status_t spsyrk_host_tril(spsyrk_session_t* session, int64_t m
     HOST_TRY(acquire(s, 1, up256(cn * 4) + up256(cn * s->sv)));
     s->d_c_colidx = s->block[1];
     s->d_c_vals = static_cast<char*>(s->block[1]) + up256(cn * 4);
-    HOST_ST(spsyrk_numeric(s->plan, (const int64_t*)s->d_c_rowptr, (int32_t*)s->d_c_colidx, s->d_c_vals, s->stream));
-    if (s->nnz_c > 0) {
-        HOST_TRY(cudaMemcpyAsync(h_c_colidx, s->d_c_colidx, (size_t)s->nnz_c * 4, cudaMemcpyDeviceToHost, s->stream));
-        HOST_TRY(cudaMemcpyAsync(h_c_vals, s->d_c_vals, (size_t)s->nnz_c * s->sv, cudaMemcpyDeviceToHost, s->stream));
+    if (s->blocks <= 1) {
+        HOST_ST(spsyrk_numeric(s->plan, (const int64_t*)s->d_c_rowptr, (int32_t*)s->d_c_colidx, s->d_c_vals, s->stream));
+        if (s->nnz_c > 0) {
+            HOST_TRY(cudaMemcpyAsync(h_c_colidx, s->d_c_colidx, (size_t)s->nnz_c * 4, cudaMemcpyDeviceToHost, s->stream));
+            HOST_TRY(cudaMemcpyAsync(h_c_vals, s->d_c_vals, (size_t)s->nnz_c * s->sv, cudaMemcpyDeviceToHost, s->stream));
+        }
+        HOST_TRY(cudaStreamSynchronize(s->stream));
+        release(s);
+        return SPSYRK_OK;
     }
-    HOST_TRY(cudaStreamSynchronize(s->stream));
+    HOST_TRY(cudaStreamCreate(&s->copy_stream));
+    cudaEvent_t done[HOST_MAX_BLOCKS] = {};
+    spsyrk_status_t st = SPSYRK_OK;
+    for (int b = 0; b < s->blocks && st == SPSYRK_OK; ++b) {
+        st = spsyrk_numeric_rows(s->plan, s->block_row[b], s->block_row[b + 1], (const int64_t*)s->d_c_rowptr, (int32_t*)s->d_c_colidx,
+                                 s->d_c_vals, s->stream);
+        if (st != SPSYRK_OK) break;
+        const int64_t o0 = s->block_off[b], cnt = s->block_off[b + 1] - o0;
+        if (cnt <= 0) continue;
+        if (cudaEventCreateWithFlags(&done[b], cudaEventDisableTiming) != cudaSuccess || cudaEventRecord(done[b], s->stream) != cudaSuccess ||
+            cudaStreamWaitEvent(s->copy_stream, done[b], 0) != cudaSuccess ||
+            cudaMemcpyAsync(h_c_colidx + o0, (const int32_t*)s->d_c_colidx + o0, (size_t)cnt * 4, cudaMemcpyDeviceToHost, s->copy_stream) != cudaSuccess ||
+            cudaMemcpyAsync((char*)h_c_vals + (size_t)o0 * s->sv, (const char*)s->d_c_vals + (size_t)o0 * s->sv, (size_t)cnt * s->sv,
+                            cudaMemcpyDeviceToHost, s->copy_stream) != cudaSuccess)
+            st = SPSYRK_ERR_CUDA;
+    }
+    if (cudaStreamSynchronize(s->stream) != cudaSuccess || cudaStreamSynchronize(s->copy_stream) != cudaSuccess) st = st == SPSYRK_OK ? SPSYRK_ERR_CUDA : st;
+    for (int b = 0; b < HOST_MAX_BLOCKS; ++b)
+        if (done[b]) cudaEventDestroy(done[b]);
     release(s);
-    return SPSYRK_OK;
+    return st;
 }

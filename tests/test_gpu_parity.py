@@ -93,6 +93,32 @@ def test_rmat_unpermuted_and_row_classes(B):
     assert (seen > 0).all(), f"row classes not all exercised: {seen}"
 
 
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_numeric_by_row_blocks(B, idx, mode):
+    """spsyrk_numeric_rows over a partition of the rows fills the same arrays as one spsyrk_numeric."""
+    a = W.small(idx)
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, mode, 0, a.m)
+    cuts = [0, 1, a.m // 5, a.m // 5, a.m // 2 + 3, a.m - 1, a.m]          # an empty block among them
+    for item_map in (False, True):
+        plan = B.spsyrk_plan(a.m, a.n, *dev(a), mode=mode)
+        B.spsyrk_plan_lend_map(plan, B._workspace(B.spsyrk_plan_map_bytes(plan), torch.device("cuda")) if item_map else None)
+        c_rowptr = torch.empty(a.m + 1, dtype=torch.int64, device="cuda")
+        nnz = B.spsyrk_symbolic(plan, c_rowptr)
+        c_colidx = torch.full((nnz,), -7, dtype=torch.int32, device="cuda")
+        c_vals = torch.zeros(nnz, dtype=torch.from_numpy(a.vals).dtype, device="cuda")
+        rp = c_rowptr.cpu().numpy()
+        for r0, r1 in zip(cuts[:-1], cuts[1:]):
+            B.spsyrk_numeric_rows(plan, r0, r1, c_rowptr, c_colidx, c_vals)
+            torch.cuda.synchronize()
+            got = c_colidx.cpu().numpy()
+            assert np.array_equal(got[:rp[r1]], ref.colidx[:rp[r1]]) and np.all(got[rp[r1]:] == -7)   # nothing beyond the block
+        check_values(c_vals.cpu().numpy(), ref, a.vals.dtype)
+        with pytest.raises(B.SpsyrkError):
+            B.spsyrk_numeric_rows(plan, 0, a.m + 1, c_rowptr, c_colidx, c_vals)
+        B.spsyrk_destroy(plan)
+
+
 @pytest.mark.parametrize("idx", [2, 3, 5])
 def test_row_tiles_concatenate(B, idx):
     a = W.small(idx)
