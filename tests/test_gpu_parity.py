@@ -119,6 +119,36 @@ def test_numeric_by_row_blocks(B, idx, mode):
         B.spsyrk_destroy(plan)
 
 
+@pytest.mark.parametrize("idx", [1, 3])
+def test_numeric_replays_from_a_cuda_graph(B, idx):
+    """The numeric pass makes no host round trip, so a caller can capture it into a CUDA graph and replay it."""
+    a = W.small(idx)
+    rp, ci, v = dev(a)
+    plan = B.spsyrk_plan(a.m, a.n, rp, ci, v)
+    B.spsyrk_plan_lend_map(plan, B._workspace(B.spsyrk_plan_map_bytes(plan), torch.device("cuda")))
+    c_rowptr = torch.empty(a.m + 1, dtype=torch.int64, device="cuda")
+    nnz = B.spsyrk_symbolic(plan, c_rowptr)
+    c_colidx = torch.empty(nnz, dtype=torch.int32, device="cuda")
+    c_vals = torch.empty(nnz, dtype=v.dtype, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        B.spsyrk_numeric(plan, c_rowptr, c_colidx, c_vals)          # warm-up outside the capture (function attributes)
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        B.spsyrk_numeric(plan, c_rowptr, c_colidx, c_vals)
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, 0, 0, a.m)
+    for _ in range(2):
+        c_vals.zero_()
+        c_colidx.fill_(-1)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(c_colidx.cpu().numpy(), ref.colidx)
+        check_values(c_vals.cpu().numpy(), ref, a.vals.dtype)
+    B.spsyrk_destroy(plan)
+
+
 @pytest.mark.parametrize("idx", [2, 3, 5])
 def test_row_tiles_concatenate(B, idx):
     a = W.small(idx)
