@@ -120,7 +120,7 @@ def class_of_rows(light_work, deg, work):
     """The library's row classes, recomputed on the host for the roofline's byte counts: light rows (at most 32
     nonzeros) are classed by `light_work` (their products without the diagonal ones in lower-triangle mode)."""
     cls = np.full(work.shape, 7, dtype=np.int8)
-    cls[work <= 8192] = 6
+    cls[work <= 32768] = 6
     light = (deg <= 32) & (light_work <= 512)
     for c, hi in ((5, 512), (4, 256), (3, 128), (2, 64), (1, 32)):
         cls[light & (light_work <= hi)] = c

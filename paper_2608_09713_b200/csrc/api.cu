@@ -21,7 +21,7 @@ void note_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); 
 namespace {
 
 constexpr size_t ALIGN = 256;
-constexpr int64_t BLOCK_CLASS_MAX_WORK = 8192;  // class 6 (256-thread CTA) up to here, class 7 above
+constexpr int64_t BLOCK_CLASS_MAX_WORK = 32768;  // class 6 (block class) up to here, class 7 above
 constexpr uint32_t ROW_CHUNK_BITS_MAX_NUMERIC = 1u << 18;
 constexpr uint32_t ROW_CHUNK_BITS_MAX_SYMBOLIC = 1u << 20;
 constexpr int TRANSPOSE_RADIX_BITS = 8;
@@ -616,7 +616,7 @@ spsyrk_status_t numeric_typed(spsyrk_plan_s* pl, int32_t* c_colidx, void* c_vals
     if (pl->map_filled) launch_numeric_map_all<V>(pl, c_colidx, c_vals, st);
     else if (pl->key64) launch_numeric_warp_all<V, uint64_t>(pl, c_colidx, c_vals, st);
     else launch_numeric_warp_all<V, uint32_t>(pl, c_colidx, c_vals, st);
-    spsyrk_status_t s = launch_numeric_cta<V, 256>(pl, 6, BLOCK_ACC_SLOTS, c_colidx, c_vals, st);
+    spsyrk_status_t s = launch_numeric_cta<V, 512>(pl, 6, BLOCK_ACC_SLOTS, c_colidx, c_vals, st);
     if (s != SPSYRK_OK) return s;
     mark(pl, pl->ev_num, 7, st);
     s = launch_numeric_cta<V, 1024>(pl, 7, 0u, c_colidx, c_vals, st);

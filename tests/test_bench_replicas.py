@@ -38,7 +38,7 @@ def test_single_process_needs_no_process_group():
     import bench
     assert bench.max_over_ranks(3.5) == 3.5
     assert bench.whole_job_rate(10.0, 1, 1000.0) == 10.0
-    work = torch.tensor([0, 10, 40, 600, 20000, 36]).numpy()
+    work = torch.tensor([0, 10, 40, 600, 40000, 36]).numpy()
     deg = torch.tensor([0, 3, 5, 40, 9, 5]).numpy()
     w = bench.class_of_rows(work, deg, work)
     assert list(w) == [0, 1, 2, 6, 7, 2]

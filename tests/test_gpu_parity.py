@@ -720,10 +720,10 @@ def test_plan_partition(B, idx):
 # ------------------------------------------------------------------ rows exactly at the class boundaries
 def test_rows_at_every_class_boundary(B):
     """One column shared by all rows: row i has exactly i + 1 partial products and i + 1 output entries,
-    so consecutive rows walk through every class boundary (32|33, 64|65, ..., 512|513, 8192|8193).
+    so consecutive rows walk through every class boundary (32|33, 64|65, ..., 512|513, 32768|32769).
     Structure by closed form for every row, values (single products, exact) for every entry, and rows
     around the boundaries against the oracle."""
-    m = 16500
+    m = 33000
     rng = np.random.default_rng(3)
     vals = rng.standard_normal(m)
     a = W.CSR(m, 1, np.arange(m + 1, dtype=np.int64), np.zeros(m, dtype=np.int32), vals)
@@ -734,13 +734,17 @@ def test_rows_at_every_class_boundary(B):
         work, classes = B.spsyrk_plan_stats(plan)
         assert work == m * (m + 1) // 2
         # a light row is classed by its products without the diagonal one (row i has i of them here)
-        assert classes == [0, 33, 32, 64, 128, 256, 8192 - 513, m - 8192]
-        rows = torch.repeat_interleave(torch.arange(m, device="cuda"), torch.arange(1, m + 1, device="cuda"))
-        cols = torch.arange(ci.numel(), device="cuda") - rp[:-1][rows]
-        assert torch.equal(ci.long(), cols)
+        assert classes == [0, 33, 32, 64, 128, 256, 32768 - 513, m - 32768]
         v = torch.from_numpy(vals).cuda()
-        assert torch.equal(cv, v[rows] * v[cols])             # one product per entry: no rounding to differ in
-        for r in (0, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257, 511, 512, 513, 8191, 8192, m - 1):
+        for r0 in range(0, m, 6000):                          # row blocks: the whole triangle at once would take tens of GB
+            r1 = min(r0 + 6000, m)
+            lo, hi = int(rp[r0]), int(rp[r1])
+            rows = torch.repeat_interleave(torch.arange(r0, r1, device="cuda"), torch.arange(r0 + 1, r1 + 1, device="cuda"))
+            cols = torch.arange(lo, hi, device="cuda") - rp[:-1][rows]
+            assert torch.equal(ci[lo:hi].long(), cols)
+            assert torch.equal(cv[lo:hi], v[rows] * v[cols])  # one product per entry: no rounding to differ in
+            del rows, cols
+        for r in (0, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257, 511, 512, 513, 8191, 8192, 32766, 32767, 32768, m - 1):
             ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, oracle.TRIL, r, r + 1)
             lo, hi = int(rp[r]), int(rp[r + 1])
             assert np.array_equal(ci[lo:hi].cpu().numpy(), ref.colidx)
@@ -794,13 +798,13 @@ def test_binary_matrix_with_heavy_columns(B, dtype, mode):
 
 # ------------------------------------------------ heavy rows beyond one bitmap chunk (more than 2^20 rows)
 def _hub_matrix(dtype):
-    """Three uniform columns per row, one column stored in 9000 scattered rows and three rows of 40
+    """Three uniform columns per row, one column stored in 36000 scattered rows and three rows of 40
     nonzeros near the end, with more than 2^20 rows: the heavy rows sit at high row indices, so their
     output range spans several bitmap chunks of the one-CTA-per-row kernels in both passes."""
     m = n = (1 << 20) + 1000
     rng = np.random.default_rng(77)
     cols = rng.integers(0, n, size=(m, 3))
-    hub_rows = np.sort(rng.choice(m, size=9000, replace=False))
+    hub_rows = np.sort(rng.choice(m, size=36000, replace=False))
     wide_rows = np.array([m - 700, m - 350, m - 2])
     lists = {}
     for r in hub_rows:
@@ -847,7 +851,7 @@ def test_heavy_rows_beyond_one_chunk(B, dtype, mode):
     cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
     # rows of every kind: hub rows early (short prefix), in the middle of the block class (one and several
     # accumulator tiles), in the large class, the rows with more than 32 nonzeros, and a few light neighbours
-    picks = [hub_rows[10], hub_rows[600], hub_rows[3000], hub_rows[5000], hub_rows[8000], hub_rows[8500], hub_rows[-1],
+    picks = [hub_rows[10], hub_rows[600], hub_rows[3000], hub_rows[5000], hub_rows[8500], hub_rows[20000], hub_rows[33500], hub_rows[-1],
              *wide_rows, hub_rows[-1] - 1 if hub_rows[-1] - 1 not in hub_rows else hub_rows[-1] + 1, a.m - 1]
     for r in picks:
         r = int(r)
