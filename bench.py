@@ -608,7 +608,7 @@ def full_variant(a, args, line, ctx):
     B, buf, ev = ctx["B"], ctx["buf"], ctx["ev"]
     d_rowptr, d_colidx, d_vals = ctx["d"]
     phases, sv, nnz_c = ctx["phases"], ctx["sv"], ctx["nnz_c"]
-    buf.pop("f", None); buf.pop("mirror_ws", None)
+    f_mirror = buf.pop("f", None); buf.pop("mirror_ws", None)   # F of the last timed step, for the comparison below
     torch.cuda.empty_cache()
     if args.no_full:
         return
@@ -621,7 +621,10 @@ def full_variant(a, args, line, ctx):
         B.spsyrk_plan_lend_map(fplan, fmap)
     fw, _ = B.spsyrk_plan_stats(fplan)
     tt = []
+    mirror_check = None
     for it in range(3):
+        if it == 1:
+            f_mirror = None  # (no cache flush here: the timed iterations reuse the blocks the first one allocated)
         e0 = ev()
         frp = torch.empty(a.m + 1, dtype=torch.int64, device="cuda")
         fn = B.spsyrk_symbolic(fplan, frp)
@@ -632,6 +635,18 @@ def full_variant(a, args, line, ctx):
         e2 = ev()
         torch.cuda.synchronize()
         tt.append((e0.elapsed_time(e1), e1.elapsed_time(e2)))
+        if it == 0 and f_mirror is not None and not args.no_verify:
+            # the mirrored lower triangle against the full product computed directly: same structure bit for bit,
+            # values within the workload's tolerance (the two halves of the full product sum in their own orders)
+            same = bool(torch.equal(f_mirror[0], frp)) and bool(torch.equal(f_mirror[1][:fn], fci[:fn]))
+            worst = None
+            if same and fn > 0:
+                x, y = f_mirror[2][:fn], fcv[:fn]
+                if x.dtype.is_floating_point:
+                    worst = float(((x - y).abs() / torch.maximum(x.abs(), y.abs()).clamp_min(1e-300)).max())
+                else:
+                    worst = float((x != y).sum())
+            mirror_check = {"structure_identical": same, "max_relative_difference_of_values": worst, "entries": int(fn)}
         del frp, fci, fcv
     fs, fnum = (float(np.mean([t[i] for t in tt[1:]])) for i in (0, 1))
     line["full_variant"] = {"multiply_adds": fw, "nnz": fn, "symbolic_ms": fs, "numeric_ms": fnum,
@@ -639,6 +654,8 @@ def full_variant(a, args, line, ctx):
                             "tril_speedup_symbolic_plus_numeric": (fs + fnum) / (phases["symbolic"] + phases["numeric"]),
                             "full_direct_vs_tril_plus_mirror": ((fs + fnum) / (phases["symbolic"] + phases["numeric"] + phases["mirror"])
                                                                 if ctx["do_mirror"] else None)}
+    if mirror_check is not None:
+        line["full_variant"]["mirror_equals_full_product"] = mirror_check
     del fplan, fmap
     torch.cuda.empty_cache()
 
