@@ -486,6 +486,25 @@ def roofline_and_variants(a, args, line, ctx, headline):
         sb = nnz_c * (4 + sv) + 8 * (a.m + 1) + 2 * a.m * sv
         sm = float(np.mean(st_[1:]))
         line["symv"] = {"ms": sm, "bytes": int(sb), "gbs": sb / (sm / 1e3) / 1e9, "frac_of_peak": sb / (sm / 1e3) / 1e9 / peak}
+        if not args.no_verify:
+            # whole-matrix check that needs no oracle: C_L x + C_L^T x - D x must equal A (A^T x) for a random x
+            # (Section V-F); the right-hand side from plain tensor operations on A, in double
+            gen = torch.Generator(device="cuda")
+            gen.manual_seed(20260807)
+            x64 = torch.rand(a.m, dtype=torch.float64, device="cuda", generator=gen) - 0.5
+            B.spsyrk_symv(a.m, keep["c"][0], keep["c"][1], keep["c"][2], x64.to(d_vals.dtype), yv)
+            xq = x64.to(d_vals.dtype).double()   # the vector the kernel saw
+            rows = torch.repeat_interleave(torch.arange(a.m, device="cuda"), d_rowptr[1:] - d_rowptr[:-1])
+            cols = d_colidx.long()
+            v64 = d_vals.double()
+            z = torch.zeros(a.n, dtype=torch.float64, device="cuda").index_add_(0, cols, v64 * xq[rows])
+            y_ref = torch.zeros(a.m, dtype=torch.float64, device="cuda").index_add_(0, rows, v64 * z[cols])
+            za = torch.zeros(a.n, dtype=torch.float64, device="cuda").index_add_(0, cols, v64.abs() * xq[rows].abs())
+            scale = torch.zeros(a.m, dtype=torch.float64, device="cuda").index_add_(0, rows, v64.abs() * za[cols])
+            worst = float(((yv.double() - y_ref).abs() / scale.clamp_min(1e-300)).max())
+            tol = 1e-12 if sv == 8 else 1e-5
+            line["symv"]["identity_with_A_At_x"] = {"max_scaled_error": worst, "tolerance": tol, "ok": bool(worst <= tol)}
+            del x64, xq, rows, cols, v64, z, y_ref, za, scale
         del xv, yv
         pcols = 8
         xm = torch.ones((a.m, pcols), dtype=d_vals.dtype, device="cuda")
