@@ -60,6 +60,34 @@ def test_random_matrices_through_every_entry_point(B, seed):
         assert np.array_equal(rp.cpu().numpy(), ref.rowptr)
         assert np.array_equal(ci.cpu().numpy(), ref.colidx)
         check_values(cv.cpu().numpy(), ref, dtype)
+        if r1 > r0:                                           # the same rows again, block by block
+            cuts = sorted({r0, r1, *(int(x) for x in rng.integers(r0, r1 + 1, size=3))})
+            crp = torch.empty(r1 - r0 + 1, dtype=torch.int64, device="cuda")
+            nn = B.spsyrk_symbolic(plan, crp)
+            cci = torch.full((max(nn, 1),), -3, dtype=torch.int32, device="cuda")
+            ccv = torch.zeros(max(nn, 1), dtype=cv.dtype, device="cuda")
+            for x0, x1 in zip(cuts[:-1], cuts[1:]):
+                B.spsyrk_numeric_rows(plan, x0, x1, crp, cci, ccv)
+            assert torch.equal(cci[:nn], ci)
+            check_values(ccv[:nn].cpu().numpy(), ref, dtype)
+        if rng.random() < 0.5:                                # a block of the product anywhere
+            b0 = int(rng.integers(0, m)); b1 = int(rng.integers(b0, m + 1))
+            s0 = int(rng.integers(0, m)); s1 = int(rng.integers(s0, m + 1))
+            bmode = int(rng.integers(0, 2))
+            bplan = B.spsyrk_plan(a.m, a.n, *d, mode=bmode)
+            B.spsyrk_plan_set_block(bplan, b0, b1, s0, s1)
+            brp, bci, bcv, _ = B.tril_syrk(a.m, a.n, *d, plan=bplan)
+            bref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, bmode, b0, b1)
+            keep = (bref.colidx >= s0) & (bref.colidx < s1)
+            rows = np.repeat(np.arange(b1 - b0), np.diff(bref.rowptr))
+            erp = np.zeros(b1 - b0 + 1, dtype=np.int64)
+            np.cumsum(np.bincount(rows[keep], minlength=b1 - b0), out=erp[1:])
+            assert np.array_equal(brp.cpu().numpy(), erp) and np.array_equal(bci.cpu().numpy(), bref.colidx[keep])
+
+            class Kept:
+                vals, absvals = bref.vals[keep], bref.absvals[keep]
+            check_values(bcv.cpu().numpy(), Kept, dtype)
+            B.spsyrk_destroy(bplan)
         if mode != 0 or (r0, r1) != (0, m):
             continue
         f = B.spsyrk_mirror(m, rp, ci, cv)
