@@ -471,6 +471,7 @@ def roofline_and_variants(a, args, line, ctx, headline):
     if not headline:
         del keep
         full_variant(a, args, line, ctx)
+        one_pass_variant(a, args, line, ctx)
         return
     # ---- consuming the triangle directly: y = C_L x + C_L^T x - D x and Y = C X (floating-point workloads)
     if not is_int:
@@ -566,6 +567,7 @@ def roofline_and_variants(a, args, line, ctx, headline):
         del pm
     del keep
     full_variant(a, args, line, ctx)
+    one_pass_variant(a, args, line, ctx)
     if args.no_full:
         return
     # ---- a half-block product of the local computation: rows of the second half against the
@@ -618,6 +620,49 @@ def roofline_and_variants(a, args, line, ctx, headline):
                                  "accumulate_ms": float(pm[4]), "accumulate_bytes": int(ab),
                                  "accumulate_gbs": ab / (float(pm[4]) / 1e3) / 1e9,
                                  "accumulate_frac_of_peak": ab / (float(pm[4]) / 1e3) / 1e9 / peak}
+    torch.cuda.empty_cache()
+
+
+def one_pass_variant(a, args, line, ctx):
+    """The one-pass mode (slots sized by the work estimate, counts found while computing, compaction) beside the
+    two passes of the timed step: the same C_L, the column lists gathered once."""
+    import torch
+    B, ev = ctx["B"], ctx["ev"]
+    d_rowptr, d_colidx, d_vals = ctx["d"]
+    phases, sv, nnz_c = ctx["phases"], ctx["sv"], ctx["nnz_c"]
+    if args.no_full:
+        return
+    if ctx.get("is_int") and not args.separate_jaccard:
+        line["one_pass"] = {"skipped": "the timed step writes the similarities with the counts; the one-pass mode does not"}
+        return
+    if 2.2 * nnz_c * (4 + sv) > 60e9:
+        line["one_pass"] = {"skipped": "slot and result buffers together would take about %.0f GB" % (2.2 * nnz_c * (4 + sv) / 1e9)}
+        return
+    plan = B.spsyrk_plan(a.m, a.n, d_rowptr, d_colidx, d_vals, mode=B.TRIL)
+    tt = []
+    slots = nnz = 0
+    for it in range(3):
+        e0 = ev()
+        slots = B.spsyrk_onepass_slots(plan)
+        s_col = torch.empty(max(slots, 1), dtype=torch.int32, device="cuda")
+        s_val = torch.empty(max(slots, 1), dtype=d_vals.dtype, device="cuda")
+        c_rowptr = torch.empty(a.m + 1, dtype=torch.int64, device="cuda")
+        e1 = ev()
+        nnz = B.spsyrk_onepass_numeric(plan, s_col, s_val, c_rowptr)
+        c_col = torch.empty(max(nnz, 1), dtype=torch.int32, device="cuda")
+        c_val = torch.empty(max(nnz, 1), dtype=d_vals.dtype, device="cuda")
+        e2 = ev()
+        B.spsyrk_onepass_compact(plan, c_rowptr, nnz, s_col, s_val, c_col, c_val)
+        e3 = ev()
+        torch.cuda.synchronize()
+        tt.append((e0.elapsed_time(e1), e1.elapsed_time(e2), e2.elapsed_time(e3)))
+        del s_col, s_val, c_rowptr, c_col, c_val
+    sl, nu, co = (float(np.mean([t[i] for t in tt[1:]])) for i in (0, 1, 2))
+    line["one_pass"] = {"slots_ms": sl, "numeric_ms": nu, "compact_ms": co, "total_ms": sl + nu + co, "four_array_form_ms": sl + nu,
+                        "two_pass_ms": phases["symbolic"] + phases["numeric"], "slot_entries": int(slots), "nnz": int(nnz),
+                        "slot_entries_over_nnz": slots / max(nnz, 1)}
+    assert nnz == nnz_c, "the one-pass mode and the symbolic pass disagree on nnz(C_L)"
+    B.spsyrk_destroy(plan)
     torch.cuda.empty_cache()
 
 
@@ -753,7 +798,7 @@ def run_ours(args):
             if cx is not None:
                 cx["buf"].clear(); cx["results"].clear(); cx.clear()
             keep = ("value", "ms_per_step", "dtype", "config", "nnz_per_s", "phases_ms", "phases_ms_median", "step_ms", "class_rows",
-                    "numeric_class_ms", "roofline", "numeric_pass", "mirror_pass", "full_variant", "clocks", "verified", "workspace")
+                    "numeric_class_ms", "roofline", "numeric_pass", "mirror_pass", "full_variant", "one_pass", "clocks", "verified", "workspace")
             others[f"config_{w}"] = {k: ro[k] for k in keep if k in ro}
             del aw, ro, cx
             B_.spsyrk_host_release_cache()

@@ -169,6 +169,32 @@ spsyrk_status_t spsyrk_numeric_rows(spsyrk_plan_t plan, int64_t row_begin, int64
                                     void *cuda_stream);
 
 /*
+ * One-pass mode: C_L without a separate symbolic pass, for callers that can afford a second, slightly larger
+ * output buffer.  Every light row gets a slot sized by the number of its partial products (an upper bound of its
+ * entries; the heavy rows, which find their structure in bitmaps anyway, get exact slots), the numeric kernel
+ * that sorts a row's products computes the row into its slot and reports its count, and the rows are then moved
+ * to their places.  The column lists are gathered once instead of twice.
+ *   1. spsyrk_onepass_slots: *slot_entries = entries the slot buffers need (>= nnz(C_L); synchronises).
+ *   2. spsyrk_onepass_numeric: fills d_slot_colidx / d_slot_vals (slot_entries entries each), writes
+ *      d_c_rowptr[rows + 1] and *nnz_out (synchronises).
+ *   3. spsyrk_onepass_compact: copies the rows into d_c_colidx / d_c_vals (nnz entries).  Asynchronous.
+ *      Optional: after step 2 the slot buffers already hold C_L in the four-array form of CSR (row begin and
+ *      row end given separately): row r occupies [b[r], b[r] + d_c_rowptr[r + 1] - d_c_rowptr[r]) of the slot
+ *      buffers with b = the rows + 1 offsets spsyrk_onepass_row_begin copies out; a consumer that accepts that
+ *      form skips step 3 and the second buffer.
+ * The result equals that of spsyrk_symbolic + spsyrk_numeric (same summation order for the light rows).
+ * Not available for the full-output mode over the whole column range (NOT_IMPLEMENTED) nor together with
+ * spsyrk_plan_set_jaccard (INVALID_ARG).  Errors: INVALID_ARG, SEQUENCE, INTERNAL, CUDA.
+ */
+spsyrk_status_t spsyrk_onepass_slots(spsyrk_plan_t plan, int64_t *slot_entries, void *cuda_stream);
+spsyrk_status_t spsyrk_onepass_numeric(spsyrk_plan_t plan, int32_t *d_slot_colidx, void *d_slot_vals,
+                                       int64_t *d_c_rowptr, int64_t *nnz_out, void *cuda_stream);
+spsyrk_status_t spsyrk_onepass_row_begin(spsyrk_plan_t plan, int64_t *d_row_begin, void *cuda_stream);
+spsyrk_status_t spsyrk_onepass_compact(spsyrk_plan_t plan, const int64_t *d_c_rowptr, int64_t nnz,
+                                       const int32_t *d_slot_colidx, const void *d_slot_vals,
+                                       int32_t *d_c_colidx, void *d_c_vals, void *cuda_stream);
+
+/*
  * spsyrk_mirror - materialise F = C_L + C_L^T - D, the full symmetric matrix, from a complete
  * (untiled or re-assembled) lower triangle (Section III-A: the full matrix, when it is needed, is
  * obtained from the stored half by a transpose; Section V-F: C = C_L + C_L^T - D).  Row i of F is row i of C_L followed by (r, c_ri) for

@@ -49,6 +49,14 @@ _lib.spsyrk_plan_lend_map.restype = _int
 _lib.spsyrk_numeric.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.spsyrk_numeric_rows.argtypes = [_vp, _i64, _i64, _vp, _vp, _vp, _vp]
 _lib.spsyrk_numeric_rows.restype = _int
+_lib.spsyrk_onepass_slots.argtypes = [_vp, _i64p, _vp]
+_lib.spsyrk_onepass_slots.restype = _int
+_lib.spsyrk_onepass_numeric.argtypes = [_vp, _vp, _vp, _vp, _i64p, _vp]
+_lib.spsyrk_onepass_numeric.restype = _int
+_lib.spsyrk_onepass_compact.argtypes = [_vp, _vp, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.spsyrk_onepass_compact.restype = _int
+_lib.spsyrk_onepass_row_begin.argtypes = [_vp, _vp, _vp]
+_lib.spsyrk_onepass_row_begin.restype = _int
 _lib.spsyrk_mirror.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_column_panel.argtypes = [_i64, _i64, _int, _vp, _vp, _vp, _i64, _i64, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
 _lib.spsyrk_accumulate.argtypes = [_i64, _int, _i64, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _i64p, _vp, _szp, _vp]
@@ -224,6 +232,53 @@ def spsyrk_numeric_rows(plan: Plan, row_begin: int, row_end: int, c_rowptr, c_co
     assert c_colidx.dtype == torch.int32 and c_vals.dtype == plan.dtype
     _check(_lib.spsyrk_numeric_rows(plan._h, int(row_begin), int(row_end), _p(c_rowptr), _p(c_colidx), _p(c_vals), _stream(stream)),
            "spsyrk_numeric_rows")
+
+
+def spsyrk_onepass_slots(plan: Plan, stream=None) -> int:
+    slots = ctypes.c_int64(0)
+    _check(_lib.spsyrk_onepass_slots(plan._h, ctypes.byref(slots), _stream(stream)), "spsyrk_onepass_slots")
+    return slots.value
+
+
+def spsyrk_onepass_numeric(plan: Plan, slot_colidx, slot_vals, c_rowptr, stream=None) -> int:
+    _dev_check(slot_colidx, slot_vals, c_rowptr)
+    assert slot_colidx.dtype == torch.int32 and slot_vals.dtype == plan.dtype and c_rowptr.dtype == torch.int64
+    nnz = ctypes.c_int64(0)
+    _check(_lib.spsyrk_onepass_numeric(plan._h, _p(slot_colidx), _p(slot_vals), _p(c_rowptr), ctypes.byref(nnz), _stream(stream)),
+           "spsyrk_onepass_numeric")
+    return nnz.value
+
+
+def spsyrk_onepass_row_begin(plan: Plan, row_begin, stream=None):
+    _dev_check(row_begin)
+    assert row_begin.dtype == torch.int64 and row_begin.numel() >= plan.rows + 1
+    _check(_lib.spsyrk_onepass_row_begin(plan._h, _p(row_begin), _stream(stream)), "spsyrk_onepass_row_begin")
+    return row_begin
+
+
+def spsyrk_onepass_compact(plan: Plan, c_rowptr, nnz, slot_colidx, slot_vals, c_colidx, c_vals, stream=None):
+    _dev_check(c_rowptr, slot_colidx, slot_vals, c_colidx, c_vals)
+    _check(_lib.spsyrk_onepass_compact(plan._h, _p(c_rowptr), int(nnz), _p(slot_colidx), _p(slot_vals), _p(c_colidx), _p(c_vals),
+                                       _stream(stream)), "spsyrk_onepass_compact")
+
+
+def onepass_syrk(plan: Plan, stream=None, compact=True):
+    """C_L through the one-pass mode: slots -> numeric into the slots -> compaction.  Returns (c_rowptr, c_colidx, c_vals);
+    with compact=False the four-array form (row_begin, c_rowptr, slot_colidx, slot_vals): row r is
+    slot_*[row_begin[r] : row_begin[r] + c_rowptr[r + 1] - c_rowptr[r]]."""
+    dev = plan._keep["a"][0].device
+    slots = spsyrk_onepass_slots(plan, stream)
+    s_col = torch.empty(max(slots, 1), dtype=torch.int32, device=dev)
+    s_val = torch.empty(max(slots, 1), dtype=plan.dtype, device=dev)
+    c_rowptr = torch.empty(plan.rows + 1, dtype=torch.int64, device=dev)
+    nnz = spsyrk_onepass_numeric(plan, s_col, s_val, c_rowptr, stream)
+    if not compact:
+        row_begin = spsyrk_onepass_row_begin(plan, torch.empty(plan.rows + 1, dtype=torch.int64, device=dev), stream)
+        return row_begin, c_rowptr, s_col, s_val
+    c_colidx = torch.empty(max(nnz, 1), dtype=torch.int32, device=dev)
+    c_vals = torch.empty(max(nnz, 1), dtype=plan.dtype, device=dev)
+    spsyrk_onepass_compact(plan, c_rowptr, nnz, s_col, s_val, c_colidx, c_vals, stream)
+    return c_rowptr, c_colidx[:nnz], c_vals[:nnz]
 
 
 def spsyrk_destroy(plan: Plan):

@@ -73,6 +73,12 @@ struct spsyrk_plan_s {
     // spsyrk_numeric_rows: the numeric launches take only positions [sub_lo[c], sub_hi[c]) of class c's row list
     bool sub_active;
     int64_t sub_lo[NCLASS], sub_hi[NCLASS];
+    // one-pass mode (spsyrk_onepass_*): per-row slot sizes (upper bounds for the light rows), their prefix sums, and
+    // where the sorting numeric kernel reports the counts it finds
+    int32_t* ub;
+    int64_t* ub_off;
+    int32_t* cnt_out;
+    bool have_onepass;
     int64_t* host_pos;  // pinned, device-visible host memory the position search of spsyrk_numeric_rows writes into (4 * NCLASS)
     int64_t rows_cap;
     // workspace views
@@ -177,6 +183,8 @@ size_t carve(spsyrk_plan_s* pl, spsyrk_plan_s* up, void* ws, int64_t m, int64_t 
     auto facts = c.take<uint32_t>(64);  // [0..2] binary analysis, [32..63] its histogram
     auto adeg = c.take<int32_t>(std::max<int64_t>(m, 1));
     auto part_bounds = c.take<int64_t>(MAX_PARTS + 1);
+    auto ub = c.take<int32_t>(std::max<int64_t>(m, 1));
+    auto ub_off = c.take<int64_t>(items + 1);
     // full-output mode: the upper view's own per-row arrays and the second descriptor array
     uint2* desc_hi = nullptr;
     int64_t *u_work = nullptr, *u_itemoff = nullptr, *u_class_start_dev = nullptr, *hi_begin = nullptr, *work_sum = nullptr;
@@ -202,6 +210,7 @@ size_t carve(spsyrk_plan_s* pl, spsyrk_plan_s* up, void* ws, int64_t m, int64_t 
         pl->desc_hi = desc_hi; pl->cnt_tot = cnt_tot; pl->hi_begin = hi_begin; pl->work_sum = work_sum;
         pl->row_counter = row_counter; pl->gacc = gacc; pl->gslots = gslots;
         pl->work_prefix = work_prefix; pl->part_bounds = part_bounds; pl->itemoff = itemoff;
+        pl->ub = ub; pl->ub_off = ub_off;
         pl->dev.heavy_id = heavy_id; pl->dev.heavy_mask = heavy_mask; pl->facts = facts;
         pl->heavy_id = heavy_id; pl->heavy_mask = heavy_mask; pl->adeg = adeg; pl->dev.adeg = adeg;
         pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.at_rec = at_rec; pl->dev.desc = desc;
@@ -307,6 +316,7 @@ __global__ void add_work_kernel(const int64_t* __restrict__ a, const int64_t* __
 spsyrk_status_t bin_view(spsyrk_plan_s* pl, cudaStream_t st) {
     const int64_t rows = pl->dev.r1 - pl->dev.r0;
     pl->have_symbolic = false;
+    pl->have_onepass = false;
     const PlanDev& P = pl->dev;
     SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->work_total_dev, 0, sizeof(unsigned long long), st));
     if (rows > 0) {
@@ -443,7 +453,7 @@ spsyrk_status_t launch_numeric_warp_d(spsyrk_plan_s* pl, int c, int32_t* c_colid
     const int64_t want = (count + ROWS - 1) / ROWS;
     const int64_t cap = (int64_t)pl->sm_count * per_sm;
     kern<<<(unsigned)std::min(want, cap), NW * 32, smem, st>>>(pl->dev, pl->hdr + numeric_first(pl, c), count, pl->out_begin, pl->out_end,
-                                                               c_colidx, static_cast<V*>(c_vals));
+                                                               c_colidx, static_cast<V*>(c_vals), pl->cnt_out);
     note_launches(1);
     return SPSYRK_OK;
 }
@@ -668,6 +678,59 @@ spsyrk_status_t symbolic_view(spsyrk_plan_s* pl, bool with_map, cudaStream_t st)
 }
 
 }  // namespace
+
+namespace {
+// slot size of every row in the one-pass layout: light rows by the number of their partial products (an upper
+// bound of their entries; with the diagonal handled apart: products without the diagonal ones, plus the diagonal
+// entry), heavy rows by the count their own symbolic kernels just found
+__global__ void onepass_slots_kernel(PlanDev P, const uint8_t* __restrict__ cls, const int32_t* __restrict__ cnt, bool diag, int64_t rows,
+                                     int32_t* __restrict__ ub) {
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    const int c = cls[r];
+    const int64_t i = P.r0 + r;
+    const int64_t deg = P.rowptr[i + 1] - P.rowptr[i];
+    int64_t u = 0;
+    if (c >= 6) u = cnt[r];
+    else if (c >= 1) u = diag ? P.work[r] - deg + (deg > 0 ? 1 : 0) : P.work[r];
+    ub[r] = (int32_t)u;  // a light row has at most 512 + 32 products
+}
+
+// G lanes per row: row r moves from its slot to its place
+template <typename V, int G>
+__global__ void __launch_bounds__(256) onepass_compact_kernel(const int64_t* __restrict__ src_off, const int64_t* __restrict__ dst_off, int64_t rows,
+                                                              const int32_t* __restrict__ s_col, const V* __restrict__ s_val,
+                                                              int32_t* __restrict__ d_col, V* __restrict__ d_val) {
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    const int gl = threadIdx.x & (G - 1);
+    if (r >= rows) return;
+    const int64_t s0 = src_off[r], d0 = dst_off[r], len = dst_off[r + 1] - d0;
+    constexpr int UNR = 4;
+    for (int64_t p = gl; p < len; p += UNR * G) {
+        int32_t j[UNR];
+        V v[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u)
+            if (p + u * G < len) { j[u] = s_col[s0 + p + u * G]; v[u] = s_val[s0 + p + u * G]; }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u)
+            if (p + u * G < len) { d_col[d0 + p + u * G] = j[u]; d_val[d0 + p + u * G] = v[u]; }
+    }
+}
+
+template <typename V>
+void launch_onepass_compact(const spsyrk_plan_s* pl, const int64_t* dst_off, int64_t rows, int64_t nnz, const int32_t* s_col, const void* s_val,
+                            int32_t* d_col, void* d_val, cudaStream_t st) {
+    const double avg = rows > 0 ? (double)nnz / (double)rows : 0.0;
+#define COMPACT(G) \
+    onepass_compact_kernel<V, G><<<(unsigned)((rows * G + 255) / 256), 256, 0, st>>>(pl->ub_off, dst_off, rows, s_col, static_cast<const V*>(s_val), \
+                                                                                  d_col, static_cast<V*>(d_val))
+    if (avg <= 4) COMPACT(4); else if (avg <= 8) COMPACT(8); else if (avg <= 16) COMPACT(16); else COMPACT(32);
+#undef COMPACT
+    note_launches(1);
+}
+}  // namespace
+
 
 extern "C" {
 
@@ -950,6 +1013,91 @@ spsyrk_status_t spsyrk_numeric_rows(spsyrk_plan_t plan, int64_t row_begin, int64
     for (int v = 0; v < 2; ++v)
         if (views[v]) views[v]->sub_active = false;
     return s;
+}
+
+spsyrk_status_t spsyrk_onepass_slots(spsyrk_plan_t plan, int64_t* slot_entries, void* cuda_stream) {
+    if (!plan || !slot_entries) return SPSYRK_ERR_INVALID_ARG;
+    spsyrk_plan_s* pl = plan;
+    if (pl->upper_active) return SPSYRK_ERR_NOT_IMPLEMENTED;  // the two-part full-output mode keeps the two-pass route
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t rows = pl->dev.r1 - pl->dev.r0;
+    pl->have_onepass = false;
+    if (rows > 0) SPSYRK_CUDA_TRY(cudaMemsetAsync(pl->cnt, 0, (size_t)rows * sizeof(int32_t), st));
+    // heavy rows: their counts come from their own kernels (bitmaps), as in the symbolic pass
+    spsyrk_status_t s = launch_symbolic_cta<256>(pl, 6, st);
+    if (s != SPSYRK_OK) return s;
+    s = launch_symbolic_cta<1024>(pl, 7, st);
+    if (s != SPSYRK_OK) return s;
+    if (rows > 0) {
+        onepass_slots_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(pl->dev, pl->cls, pl->cnt, pl->diag, rows, pl->ub);
+        note_launches(1);
+    }
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<int32_t>(pl->ub, rows, pl->ub_off, pl->partials, st));
+    int64_t total = 0;
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(&total, pl->ub_off + rows, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
+    s = read_err(pl, st);
+    if (s != SPSYRK_OK) return s;
+    *slot_entries = total;
+    pl->have_onepass = true;
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_onepass_numeric(spsyrk_plan_t plan, int32_t* d_slot_colidx, void* d_slot_vals, int64_t* d_c_rowptr, int64_t* nnz_out,
+                                       void* cuda_stream) {
+    if (!plan || !d_c_rowptr || !nnz_out) return SPSYRK_ERR_INVALID_ARG;
+    spsyrk_plan_s* pl = plan;
+    if (!pl->have_onepass) return SPSYRK_ERR_SEQUENCE;
+    if (pl->dev.jaccard) return SPSYRK_ERR_INVALID_ARG;  // the fused similarity is written at final offsets only
+    if (pl->work_total > 0 && (!d_slot_colidx || !d_slot_vals)) return SPSYRK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t rows = pl->dev.r1 - pl->dev.r0;
+    // every row is computed into its slot; the light rows report their counts (the heavy ones have theirs already)
+    const bool map_was = pl->map_filled;
+    pl->map_filled = false;  // the kernel that sorts in the numeric pass counts as it goes
+    pl->cnt_out = pl->cnt;
+    pl->out_begin = pl->ub_off;
+    pl->out_end = pl->ub_off + 1;
+    spsyrk_status_t s;
+    switch (pl->dtype) {
+        case SPSYRK_F64: s = numeric_typed<double>(pl, d_slot_colidx, d_slot_vals, st); break;
+        case SPSYRK_F32: s = numeric_typed<float>(pl, d_slot_colidx, d_slot_vals, st); break;
+        default: s = numeric_typed<int32_t>(pl, d_slot_colidx, d_slot_vals, st); break;
+    }
+    pl->cnt_out = nullptr;
+    pl->map_filled = map_was;
+    if (s != SPSYRK_OK) return s;
+    SPSYRK_CUDA_TRY(exclusive_scan_i64<int32_t>(pl->cnt, rows, d_c_rowptr, pl->partials, st));
+    int64_t nnz = 0;
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(&nnz, d_c_rowptr + rows, sizeof(int64_t), cudaMemcpyDeviceToHost, st));
+    s = read_err(pl, st);
+    if (s != SPSYRK_OK) return s;
+    *nnz_out = nnz;
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_onepass_row_begin(spsyrk_plan_t plan, int64_t* d_row_begin, void* cuda_stream) {
+    if (!plan || !d_row_begin) return SPSYRK_ERR_INVALID_ARG;
+    if (!plan->have_onepass) return SPSYRK_ERR_SEQUENCE;
+    const int64_t rows = plan->dev.r1 - plan->dev.r0;
+    SPSYRK_CUDA_TRY(cudaMemcpyAsync(d_row_begin, plan->ub_off, (size_t)(rows + 1) * sizeof(int64_t), cudaMemcpyDeviceToDevice,
+                                    static_cast<cudaStream_t>(cuda_stream)));
+    return SPSYRK_OK;
+}
+
+spsyrk_status_t spsyrk_onepass_compact(spsyrk_plan_t plan, const int64_t* d_c_rowptr, int64_t nnz, const int32_t* d_slot_colidx,
+                                       const void* d_slot_vals, int32_t* d_c_colidx, void* d_c_vals, void* cuda_stream) {
+    if (!plan || !d_c_rowptr || nnz < 0) return SPSYRK_ERR_INVALID_ARG;
+    spsyrk_plan_s* pl = plan;
+    if (!pl->have_onepass) return SPSYRK_ERR_SEQUENCE;
+    if (nnz > 0 && (!d_slot_colidx || !d_slot_vals || !d_c_colidx || !d_c_vals)) return SPSYRK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t rows = pl->dev.r1 - pl->dev.r0;
+    if (rows > 0 && nnz > 0) {
+        if (pl->dtype == SPSYRK_F64) launch_onepass_compact<uint64_t>(pl, d_c_rowptr, rows, nnz, d_slot_colidx, d_slot_vals, d_c_colidx, d_c_vals, st);
+        else launch_onepass_compact<uint32_t>(pl, d_c_rowptr, rows, nnz, d_slot_colidx, d_slot_vals, d_c_colidx, d_c_vals, st);
+    }
+    SPSYRK_CUDA_TRY(cudaGetLastError());
+    return SPSYRK_OK;
 }
 
 spsyrk_status_t spsyrk_plan_map_bytes(spsyrk_plan_t plan, size_t* bytes) {

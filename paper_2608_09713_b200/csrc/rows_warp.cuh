@@ -100,9 +100,12 @@ struct NumericWarpSmem {
 template <typename V, int N, int G, typename Key, bool DIAG>
 __global__ void __launch_bounds__(numeric_warps(N) * 32, numeric_min_ctas(N))
 numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows, const int64_t* __restrict__ c_rowptr,
-                    const int64_t* __restrict__ c_rowend, int32_t* __restrict__ c_colidx, V* __restrict__ c_vals) {
+                    const int64_t* __restrict__ c_rowend, int32_t* __restrict__ c_colidx, V* __restrict__ c_vals,
+                    int32_t* __restrict__ cnt_out = nullptr) {
     // c_rowptr[r] / c_rowend[r]: where row r's part of the output starts and ends (c_rowend = c_rowptr + 1 unless the
-    // rows are written in two parts, see the full-output mode of the plan)
+    // rows are written in two parts, see the full-output mode of the plan).  cnt_out: the kernel counts the entries of
+    // a row itself while it merges equal column ids, so it can also serve rows whose slots were sized by an upper
+    // bound (the one-pass mode); it then reports the counts here.
     using Acc = typename AccOf<V>::type;
     using Rec = ColRec<V>;
     using SM = NumericWarpSmem<V, N>;
@@ -333,6 +336,7 @@ numeric_warp_kernel(PlanDev P, const uint4* __restrict__ hdr, int64_t nrows, con
             if (!SPSYRK_IN_RANGE((int64_t)total <= room && total <= NP - 1, P.err)) total = 0;
         }
 #endif
+        if (cnt_out && gl == 0 && h_n.z > 0) cnt_out[h_n.x] = total;
         for (int o = gl; o < total; o += G) {
             const int32_t j = (int32_t)o_j[o + (o >> 3)];
             const V cv = o_v[o + (o >> 3)];

@@ -24,7 +24,9 @@ def test_checked_build_runs_clean():
     assert probe.returncode == 0 and probe.stdout.strip() == CHECKED, probe.stderr[-2000:]
     sel = ["tests/test_gpu_parity.py::test_small_configs", "tests/test_gpu_parity.py::test_mirror",
            "tests/test_gpu_parity.py::test_rows_at_every_class_boundary", "tests/test_gpu_parity.py::test_blocks",
-           "tests/test_gpu_parity.py::test_symm", "tests/test_gpu_random.py"]
+           "tests/test_gpu_parity.py::test_symm", "tests/test_gpu_parity.py::test_one_pass_mode",
+           "tests/test_gpu_parity.py::test_numeric_by_row_blocks", "tests/test_gpu_parity.py::test_mirror_general_lower_triangles",
+           "tests/test_gpu_random.py"]
     run = subprocess.run([sys.executable, "-m", "pytest", *sel, "-m", "gpu", "-x", "-q", "-p", "no:cacheprovider"],
                          cwd=ROOT, env=env, capture_output=True, text=True, timeout=3000)
     assert run.returncode == 0, run.stdout[-4000:] + run.stderr[-2000:]

@@ -119,6 +119,43 @@ def test_numeric_by_row_blocks(B, idx, mode):
         B.spsyrk_destroy(plan)
 
 
+@pytest.mark.parametrize("idx", [1, 2, 3, 4, 5])
+def test_one_pass_mode(B, idx):
+    """Slots from the work estimate, rows computed into them with their counts found on the way, then compacted:
+    the same C_L as symbolic + numeric; also for a row range and a block of columns."""
+    a = W.small(idx)
+    d = dev(a)
+    ref = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, 0, 0, a.m)
+    plan = B.spsyrk_plan(a.m, a.n, *d)
+    rp, ci, cv = B.onepass_syrk(plan)
+    torch.cuda.synchronize()
+    assert np.array_equal(rp.cpu().numpy(), ref.rowptr) and np.array_equal(ci.cpu().numpy(), ref.colidx)
+    check_values(cv.cpu().numpy(), ref, a.vals.dtype)
+    # the four-array form the slot buffers hold before the compaction: the same rows, each in its slot
+    rb, rp4, sc, sv_ = B.onepass_syrk(plan, compact=False)
+    assert torch.equal(rp4, rp)
+    lens = rp[1:] - rp[:-1]
+    assert bool((rb[:-1] + lens <= rb[1:]).all())
+    idx = torch.repeat_interleave(rb[:-1] - rp[:-1], lens) + torch.arange(ci.numel(), device="cuda")
+    assert torch.equal(sc[idx], ci) and torch.equal(sv_[idx], cv)
+    r0, r1 = a.m // 3, a.m - 5
+    B.spsyrk_plan_set_rows(plan, r0, r1)
+    rp, ci, cv = B.onepass_syrk(plan)
+    part = oracle.syrk(a.m, a.n, a.rowptr, a.colidx, a.vals, 0, r0, r1)
+    assert np.array_equal(rp.cpu().numpy(), part.rowptr) and np.array_equal(ci.cpu().numpy(), part.colidx)
+    check_values(cv.cpu().numpy(), part, a.vals.dtype)
+    h = a.m // 2
+    B.spsyrk_plan_set_block(plan, h, a.m, 0, h)            # an off-diagonal block: no diagonal handled apart
+    rp, ci, cv = B.onepass_syrk(plan)
+    cols = oracle.transpose(a.m, a.n, a.rowptr, a.colidx, a.vals)
+    blk = oracle_block(a, oracle.TRIL, h, a.m, 0, h, cols)
+    assert np.array_equal(rp.cpu().numpy(), blk.rowptr) and np.array_equal(ci.cpu().numpy(), blk.colidx)
+    check_values(cv.cpu().numpy(), blk, a.vals.dtype)
+    fplan = B.spsyrk_plan(a.m, a.n, *d, mode=B.FULL)
+    with pytest.raises(B.SpsyrkError):
+        B.onepass_syrk(fplan)                              # the two-part full-output mode keeps the two-pass route
+
+
 @pytest.mark.parametrize("idx", [1, 3])
 def test_numeric_replays_from_a_cuda_graph(B, idx):
     """The numeric pass makes no host round trip, so a caller can capture it into a CUDA graph and replay it."""
