@@ -98,6 +98,11 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     const bool binary = P.binary != 0;
     const bool use_masks = NUMERIC && dense && binary && P.nheavy > 0;
     const unsigned long long mask_i = use_masks ? P.heavy_mask[i] : 0ull;
+    // Binary input, dense row of at most 255 nonzeros: every count is at most the row's own length, so four
+    // 8-bit counters share a 32-bit word of the accumulator tile and a tile holds four times the columns
+    // (a row of 1e5 columns is one tile: its lists are cut into column ranges once, not once per tile).
+    const bool packed = NUMERIC && !GLOBAL_ACC && std::is_same<V, int32_t>::value && dense && binary && deg <= 255u;
+    const uint32_t row_tile_slots = packed ? tile_slots * 4u : tile_slots;
 
     // One partial product: set its bit, or add it into its slot.
     auto apply = [&](auto what, auto dense_tag, uint32_t rel, Acc a, Acc v, uint32_t s0) {
@@ -108,7 +113,9 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
         } else {
             if (!SPSYRK_IN_RANGE(DENSE || (rel >> 5) < cw, P.err)) return;
             const uint32_t slot = (DENSE ? rel : rank[rel >> 5] + __popc(bits[rel >> 5] & ((1u << (rel & 31)) - 1u))) - s0;
-            if (SPSYRK_IN_RANGE(slot < tile_slots, P.err)) atomicAdd(&acc[slot], acc_mul(a, v));
+            if (!SPSYRK_IN_RANGE(slot < row_tile_slots, P.err)) return;
+            if (DENSE && packed) atomicAdd(reinterpret_cast<uint32_t*>(acc) + (slot >> 2), 1u << ((slot & 3u) * 8u));  // a product of a binary matrix is 1
+            else atomicAdd(&acc[slot], acc_mul(a, v));
         }
     };
 
@@ -273,8 +280,8 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     }
                 }
             }
-            for (uint32_t s0 = 0; s0 < tot; s0 += tile_slots) {
-                const uint32_t s1 = min(s0 + tile_slots, tot);
+            for (uint32_t s0 = 0; s0 < tot; s0 += row_tile_slots) {
+                const uint32_t s1 = min(s0 + row_tile_slots, tot);
                 const bool single_tile = (s0 == 0 && s1 == tot);
                 uint32_t jlo = c0, jhi = c1;
                 if (!single_tile && dense) {
@@ -303,7 +310,20 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     jlo = s_sel[0];
                     jhi = s_sel[1];
                 }
-                if (use_masks) {
+                if (packed) {
+                    // slot t of a dense row is column c0 + s0 + t; word w holds slots 4 w .. 4 w + 3
+                    const uint64_t* mk = P.heavy_mask + c0 + s0;
+                    uint32_t* acc32 = reinterpret_cast<uint32_t*>(acc);
+                    for (uint32_t w = tid; w < (s1 - s0 + 3u) / 4u; w += THREADS) {
+                        uint32_t word = 0;
+                        if (use_masks) {
+#pragma unroll
+                            for (uint32_t q = 0; q < 4; ++q)
+                                if (4u * w + q < s1 - s0) word |= (uint32_t)__popcll((unsigned long long)mk[4u * w + q] & mask_i) << (8u * q);
+                        }
+                        acc32[w] = word;
+                    }
+                } else if (use_masks) {
                     // slot t of a dense row is column c0 + s0 + t
                     const uint64_t* mk = P.heavy_mask + c0 + s0;
                     for (uint32_t t = tid; t < s1 - s0; t += THREADS) acc[t] = Acc(__popcll((unsigned long long)mk[t] & mask_i));
@@ -316,7 +336,8 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                 else for_each_product(ACC, NOT_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
                 for (uint32_t t = tid; t < s1 - s0; t += THREADS) {
                     if (!SPSYRK_IN_RANGE(ob + s0 + t < out_end, P.err)) continue;
-                    const V cv = (V)(GLOBAL_ACC ? __ldcg(acc + t) : acc[t]);
+                    const V cv = packed ? (V)((reinterpret_cast<const uint32_t*>(acc)[t >> 2] >> ((t & 3u) * 8u)) & 0xffu)
+                                        : (V)(GLOBAL_ACC ? __ldcg(acc + t) : acc[t]);
                     c_vals[ob + s0 + t] = cv;
                     if constexpr (std::is_same<V, int32_t>::value) {
                         if (P.jaccard) {
