@@ -816,9 +816,12 @@ def test_binary_matrix_with_heavy_columns(B, dtype, mode):
     mask[:, 17] = True
     for k, dens in zip(rng.choice(n, size=90, replace=False), np.linspace(0.09, 0.9, 90)):
         mask[:, k] |= rng.random(m) < dens
+    for r in (5, 1500, 2990):                                # rows of more than 255 nonzeros: their counts need full words,
+        mask[r, rng.choice(n, size=400, replace=False)] = True   # the other rows pack four 8-bit counters per word
     rr, cc = np.nonzero(mask)
     rowptr = np.zeros(m + 1, dtype=np.int64)
     np.cumsum(np.bincount(rr, minlength=m), out=rowptr[1:])
+    assert np.diff(rowptr).max() > 255 and np.median(np.diff(rowptr)) < 255
     a = W.CSR(m, n, rowptr, cc.astype(np.int32), np.ones(cc.size, dtype=dtype))
     (rp, ci, cv), ref, plan = run_and_compare(B, a, mode)
     if dtype == np.int32 and mode == 0:
