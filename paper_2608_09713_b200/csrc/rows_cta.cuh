@@ -265,10 +265,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
         }
         if (NUMERIC) {
             const int64_t ob = out_base + total_cnt;
-            if (dense) {
-                for (uint32_t t = tid; t < tot; t += THREADS)
-                    if (SPSYRK_IN_RANGE(ob + t < out_end, P.err)) c_colidx[ob + t] = (int32_t)(c0 + t);
-            } else {
+            if (!dense) {  // (a dense row writes its column ids, c0 + slot, with its values below)
                 // column ids straight from the bitmap
                 for (uint32_t w = tid; w < cwa; w += THREADS) {
                     uint32_t b = bits[w], r = rank[w];
@@ -339,6 +336,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     const V cv = packed ? (V)((reinterpret_cast<const uint32_t*>(acc)[t >> 2] >> ((t & 3u) * 8u)) & 0xffu)
                                         : (V)(GLOBAL_ACC ? __ldcg(acc + t) : acc[t]);
                     c_vals[ob + s0 + t] = cv;
+                    if (dense) c_colidx[ob + s0 + t] = (int32_t)(c0 + s0 + t);
                     if constexpr (std::is_same<V, int32_t>::value) {
                         if (P.jaccard) {
                             // J = c / (|a_i| + |a_j| - c); the column id was written above (dense rows: it is the slot's column)
