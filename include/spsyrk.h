@@ -389,11 +389,12 @@ spsyrk_status_t spsyrk_plan_stats(spsyrk_plan_t plan, int64_t *work_total, int64
 
 /*
  * spsyrk_plan_buffers - device pointers into the plan's workspace, for inspection and tests:
- * column pointers colptr[n+1] (int64), the column lists' row ids at_row[nnz] (int32) and
- * values at_val[nnz] (plan dtype), and the per-row work w[rows] (int64).  Any may be NULL.
+ * column pointers colptr[n+1] (int64), the column lists' row ids at_row[nnz] (int32), the same
+ * entries as (row id, value) records at_rec[nnz] (8-byte values: int32 row id, 4 bytes of padding, the
+ * value; 4-byte values: int32 row id, the value), and the per-row work w[rows] (int64).  Any may be NULL.
  */
 spsyrk_status_t spsyrk_plan_buffers(spsyrk_plan_t plan, const int64_t **d_colptr, const int32_t **d_at_row,
-                                    const void **d_at_val, const int64_t **d_work);
+                                    const void **d_at_rec, const int64_t **d_work);
 
 /*
  * Measurement aids (no effect on results).

@@ -321,7 +321,8 @@ def spsyrk_launch_count() -> int:
 
 
 def spsyrk_plan_buffers(plan: Plan):
-    """Copies of the plan's column lists and work estimate as torch tensors: (colptr, at_row, at_val, work)."""
+    """Copies of the plan's column lists and work estimate as torch tensors: (colptr, at_row, at_val, work); the values
+    are taken out of the plan's (row id, value) records."""
     ptrs = [_vp() for _ in range(4)]
     _check(_lib.spsyrk_plan_buffers(plan._h, *[ctypes.byref(p) for p in ptrs]), "spsyrk_plan_buffers")
     nnz = plan._keep["a"][1].numel()
@@ -333,8 +334,9 @@ def spsyrk_plan_buffers(plan: Plan):
         return torch.as_tensor(_DevArray(ptr.value, count, _TYPESTR[dtype]), device=dev).clone()
 
     torch.cuda.synchronize()
-    return (view(ptrs[0], plan.n + 1, torch.int64), view(ptrs[1], nnz, torch.int32),
-            view(ptrs[2], nnz, plan.dtype), view(ptrs[3], plan.rows, torch.int64))
+    # a record is (row id, [padding,] value): seen as 2 * nnz elements of the value type, the values are the odd ones
+    at_val = view(ptrs[2], 2 * nnz, plan.dtype)[1::2].contiguous()
+    return (view(ptrs[0], plan.n + 1, torch.int64), view(ptrs[1], nnz, torch.int32), at_val, view(ptrs[3], plan.rows, torch.int64))
 
 
 _TYPESTR = {torch.int64: "<i8", torch.int32: "<i4", torch.float64: "<f8", torch.float32: "<f4"}

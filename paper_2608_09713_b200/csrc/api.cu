@@ -134,7 +134,6 @@ size_t carve(spsyrk_plan_s* pl, spsyrk_plan_s* up, void* ws, int64_t m, int64_t 
     const int64_t items = std::max<int64_t>(std::max(m, n), 1);
     const int64_t nb = bin_blocks(items);
     auto colptr = c.take<int64_t>(n + 1);
-    auto at_val = c.take<char>(nnz * sv);
     auto desc = c.take<uint2>(nnz);
     auto work = c.take<int64_t>(m);
     auto perm = c.take<int32_t>(m);
@@ -213,7 +212,7 @@ size_t carve(spsyrk_plan_s* pl, spsyrk_plan_s* up, void* ws, int64_t m, int64_t 
         pl->ub = ub; pl->ub_off = ub_off;
         pl->dev.heavy_id = heavy_id; pl->dev.heavy_mask = heavy_mask; pl->facts = facts;
         pl->heavy_id = heavy_id; pl->heavy_mask = heavy_mask; pl->adeg = adeg; pl->dev.adeg = adeg;
-        pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_val = at_val; pl->dev.at_rec = at_rec; pl->dev.desc = desc;
+        pl->dev.colptr = colptr; pl->dev.at_row = at_row; pl->dev.at_rec = at_rec; pl->dev.desc = desc;
         pl->dev.work = work; pl->dev.err = err;
         pl->desc_full = desc; pl->desc_blk = desc_blk;
         pl->perm = perm; pl->hdr = hdr; pl->cnt = cnt; pl->cls = cls; pl->colcnt = colcnt;
@@ -1133,11 +1132,11 @@ spsyrk_status_t spsyrk_plan_stats(spsyrk_plan_t plan, int64_t* work_total, int64
 }
 
 spsyrk_status_t spsyrk_plan_buffers(spsyrk_plan_t plan, const int64_t** d_colptr, const int32_t** d_at_row,
-                                    const void** d_at_val, const int64_t** d_work) {
+                                    const void** d_at_rec, const int64_t** d_work) {
     if (!plan) return SPSYRK_ERR_INVALID_ARG;
     if (d_colptr) *d_colptr = plan->dev.colptr;
     if (d_at_row) *d_at_row = plan->dev.at_row;
-    if (d_at_val) *d_at_val = plan->dev.at_val;
+    if (d_at_rec) *d_at_rec = plan->dev.at_rec;
     if (d_work) *d_work = plan->upper_active ? plan->work_sum : plan->dev.work;
     return SPSYRK_OK;
 }

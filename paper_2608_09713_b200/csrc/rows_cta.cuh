@@ -203,8 +203,15 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                             rel[u] = 0;
                             val[u] = Acc(0);
                             if (q[u] != 0xffffffffu) {
-                                rel[u] = (uint32_t)P.at_row[q[u]] - c0;
-                                if (WHAT == CTA_ACCUM) val[u] = binary ? Acc(1) : (Acc) static_cast<const V*>(P.at_val)[q[u]];
+                                if (WHAT == CTA_ACCUM && !binary) {
+                                    // one load brings the row id and the value (the records the light rows gather)
+                                    const ColRec<V> rec = static_cast<const ColRec<V>*>(P.at_rec)[q[u]];
+                                    rel[u] = (uint32_t)rec.j - c0;
+                                    val[u] = (Acc)rec.v;
+                                } else {
+                                    rel[u] = (uint32_t)P.at_row[q[u]] - c0;
+                                    if (WHAT == CTA_ACCUM) val[u] = Acc(1);
+                                }
                             }
                         }
 #pragma unroll
@@ -219,7 +226,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                 const uint32_t t = long_idx[li];
                 const uint32_t len = llen[t];
                 const int32_t* __restrict__ rowp = P.at_row + lstart[t];
-                const V* __restrict__ valp = static_cast<const V*>(P.at_val) + lstart[t];
+                const ColRec<V>* __restrict__ recp = static_cast<const ColRec<V>*>(P.at_rec) + lstart[t];
                 const Acc fa = WHAT == CTA_ACCUM ? la[t] : Acc(0);
                 uint32_t e = tid;
                 for (; e + (UNR - 1) * THREADS < len; e += UNR * THREADS) {
@@ -227,14 +234,26 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     Acc val[UNR];
 #pragma unroll
                     for (int u = 0; u < UNR; ++u) {
-                        rel[u] = (uint32_t)rowp[e + u * THREADS] - c0;
-                        val[u] = (WHAT == CTA_ACCUM && !binary) ? (Acc)valp[e + u * THREADS] : Acc(1);
+                        if (WHAT == CTA_ACCUM && !binary) {
+                            const ColRec<V> rec = recp[e + u * THREADS];
+                            rel[u] = (uint32_t)rec.j - c0;
+                            val[u] = (Acc)rec.v;
+                        } else {
+                            rel[u] = (uint32_t)rowp[e + u * THREADS] - c0;
+                            val[u] = Acc(1);
+                        }
                     }
 #pragma unroll
                     for (int u = 0; u < UNR; ++u) apply(what, dense_tag, rel[u], fa, val[u], s0);
                 }
-                for (; e < len; e += THREADS)
-                    apply(what, dense_tag, (uint32_t)rowp[e] - c0, fa, (WHAT == CTA_ACCUM && !binary) ? (Acc)valp[e] : Acc(1), s0);
+                for (; e < len; e += THREADS) {
+                    if (WHAT == CTA_ACCUM && !binary) {
+                        const ColRec<V> rec = recp[e];
+                        apply(what, dense_tag, (uint32_t)rec.j - c0, fa, (Acc)rec.v, s0);
+                    } else {
+                        apply(what, dense_tag, (uint32_t)rowp[e] - c0, fa, Acc(1), s0);
+                    }
+                }
             }
             __syncthreads();
         }

@@ -2,7 +2,8 @@
 // plus the per-nonzero descriptors the row kernels consume.
 //
 //   colptr[n+1]        column pointers (int64)
-//   at_row[q], at_val[q]  entries of the column lists, q in [colptr[k], colptr[k+1]) ascending by row
+//   at_row[q], at_rec[q]  entries of the column lists, q in [colptr[k], colptr[k+1]) ascending by row: the row ids
+//                      alone (what the structure passes read) and (row id, value) records (what the value passes read)
 //   desc[p] = (start, len) for nonzero p = (i, k) of A: start = colptr[k]; len = number of entries
 //             of column k with row <= i (the rank of i in the list, plus one).  "Rows j <= i of
 //             column k" is then at_row[start, start+len).  The full-output mode also keeps the rest of
@@ -11,7 +12,7 @@
 // Method: histogram of column ids and scan for colptr; then a stable LSD radix sort of the
 // nonzeros by column id with (row, value, position in A) as payload.  The nonzeros enter in row
 // order, so each column's segment comes out ascending by row; the last pass writes at_row and
-// at_val and scatters the descriptor, whose length is the entry's rank inside its column.  (The
+// at_rec and scatters the descriptor, whose length is the entry's rank inside its column.  (The
 // value travels with the element because reading it in the first pass is sequential, whereas
 // fetching it by position in the last pass is one random access per nonzero.)
 #pragma once
@@ -29,7 +30,7 @@ struct PlanDev {
     const void* vals;
     int64_t* colptr;
     int32_t* at_row;
-    void* at_val;
+    // (the values of the column lists live in the records only)
     void* at_rec;  // the same entries as interleaved (row id, value) records: ColRec<V>[nnz]
     uint2* desc;
     int64_t* work;  // per row of the range
@@ -177,7 +178,6 @@ struct EmitTransposeFinal {
     __device__ __forceinline__ void operator()(int64_t s, uint32_t k, uint32_t row, VB val, uint32_t p) const {
         const int64_t cs = P.colptr[k];
         P.at_row[s] = (int32_t)row;
-        static_cast<VB*>(P.at_val)[s] = val;  // bit copy of the value that travelled with the element
         if constexpr (sizeof(VB) == 8) static_cast<uint4*>(P.at_rec)[s] = make_uint4(row, 0u, (uint32_t)val, (uint32_t)(val >> 32));
         else static_cast<uint2*>(P.at_rec)[s] = make_uint2(row, (uint32_t)val);
         // the entries of column k with row <= i are the first rank + 1 of its list; the full-output mode also keeps
