@@ -245,7 +245,7 @@ template <int G>
 void launch_row_expand(spsyrk_plan_s* pl, cudaStream_t st) {
     const PlanDev& P = pl->dev;
     const int64_t threads = (int64_t)P.m * G;
-    row_expand_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P.rowptr, P.colidx, P.m, pl->rx_row_b, P.err);
+    row_expand_kernel<G><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(P.rowptr, P.colidx, P.m, P.n, pl->colcnt, pl->rx_row_b, P.err);
     note_launches(1);
 }
 
@@ -790,13 +790,8 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
     PLAN_TRY(cudaGetLastError());
     spsyrk_status_t s = read_err(pl, st);
     if (s != SPSYRK_OK) return fail(s);
-    // 2. transpose: column histogram and scan give colptr; explicit row ids; stable radix sort by column
-    if (nnz > 0) {
-        const unsigned hb = (unsigned)std::min<int64_t>((nnz + 255) / 256, (int64_t)pl->sm_count * 32);
-        column_histogram_kernel<<<hb, 256, 0, st>>>(d_colidx, nnz, P.n, pl->colcnt, P.err);
-        note_launches(1);
-    }
-    PLAN_TRY(exclusive_scan_i64<uint32_t>(pl->colcnt, n, P.colptr, pl->partials, st));
+    // 2. transpose: one sweep over A for the column histogram, the explicit row ids and the checks of the column
+    // ids; the histogram's scan gives colptr; stable radix sort by column
     if (nnz > 0) {
         switch (group_width(nnz, m)) {
             case 4: launch_row_expand<4>(pl, st); break;
@@ -805,6 +800,7 @@ spsyrk_status_t spsyrk_plan(spsyrk_plan_t* plan, int64_t m, int64_t n, int64_t n
             default: launch_row_expand<32>(pl, st); break;
         }
     }
+    PLAN_TRY(exclusive_scan_i64<uint32_t>(pl->colcnt, n, P.colptr, pl->partials, st));
     s = read_err(pl, st);  // synchronises; column ids are known to be in range and rows sorted from here on
     if (s != SPSYRK_OK) return fail(s);
     s = sv == 8 ? sort_by_column<uint64_t>(pl, st) : sort_by_column<uint32_t>(pl, st);

@@ -144,28 +144,22 @@ static __global__ void validate_rowptr_kernel(const int64_t* __restrict__ rowptr
     if (i == 0 && (rowptr[0] != 0 || rowptr[m] != nnz)) atomicOr(err, ERRW_BAD_ROWPTR);
 }
 
-static __global__ void column_histogram_kernel(const int32_t* __restrict__ colidx, int64_t nnz, int32_t n,
-                                        uint32_t* __restrict__ colcnt, uint32_t* err) {
-    int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (; p < nnz; p += stride) {
-        int32_t k = colidx[p];
-        if ((uint32_t)k >= (uint32_t)n) atomicOr(err, ERRW_BAD_COL);
-        else atomicAdd(&colcnt[k], 1u);
-    }
-}
-
-// G lanes per row: the explicit row id of every nonzero (the radix sort's first payload); also
-// checks that column ids are strictly ascending inside the row.
+// G lanes per row, one sweep over the nonzeros of A: the column histogram (its scan gives colptr), the explicit
+// row id of every nonzero (the radix sort's first payload), and the checks that column ids are in range and
+// strictly ascending inside the row.  The row pointers have been validated before.
 template <int G>
 static __global__ void __launch_bounds__(256) row_expand_kernel(const int64_t* __restrict__ rowptr, const int32_t* __restrict__ colidx,
-                                                                int32_t m, uint32_t* __restrict__ rowid, uint32_t* err) {
+                                                                int32_t m, int32_t n, uint32_t* __restrict__ colcnt,
+                                                                uint32_t* __restrict__ rowid, uint32_t* err) {
     const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
     const int gl = threadIdx.x & (G - 1);
     if (gid >= m) return;
     const int64_t p0 = rowptr[gid], p1 = rowptr[gid + 1];
     for (int64_t p = p0 + gl; p < p1; p += G) {
-        if (p > p0 && colidx[p - 1] >= colidx[p]) atomicOr(err, ERRW_UNSORTED);
+        const int32_t k = colidx[p];
+        if ((uint32_t)k >= (uint32_t)n) atomicOr(err, ERRW_BAD_COL);
+        else atomicAdd(&colcnt[k], 1u);
+        if (p > p0 && colidx[p - 1] >= k) atomicOr(err, ERRW_UNSORTED);
         rowid[p] = (uint32_t)gid;
     }
 }
