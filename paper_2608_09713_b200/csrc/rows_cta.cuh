@@ -18,6 +18,13 @@ namespace spsyrk {
 
 enum : int { CTA_SETBITS = 0, CTA_ACCUM = 1 };
 
+// CTAs per SM the launches are sized for (shared memory allows no more): stated so that the register allocation
+// does not trade spills for an occupancy the kernel cannot reach
+// (the counting pass holds little state: it keeps the 32 registers that let 2048 threads share an SM)
+__host__ __device__ constexpr int cta_min_blocks(int threads, bool numeric) {
+    return !numeric ? 2048 / threads : threads >= 1024 ? 1 : threads >= 512 ? 2 : 3;
+}
+
 template <typename V, int THREADS, bool NUMERIC>
 struct CtaRowSmem {
     using Acc = typename AccOf<V>::type;
@@ -36,7 +43,7 @@ struct CtaRowSmem {
 // CTAs fetch rows from a counter, so that the slice indexed by blockIdx.x is never shared.  The
 // two variants are launched over the same row list and each skips the rows of the other.
 template <typename V, int THREADS, bool NUMERIC, bool GLOBAL_ACC = false>
-__global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int32_t* __restrict__ rows,
+__global__ void __launch_bounds__(THREADS, cta_min_blocks(THREADS, NUMERIC)) rows_cta_kernel(PlanDev P, const int32_t* __restrict__ rows,
                                                            uint32_t chunk_bits, uint32_t acc_slots,
                                                            int32_t* __restrict__ cnt,
                                                            const int64_t* __restrict__ c_rowptr, const int64_t* __restrict__ c_rowend,
@@ -127,9 +134,11 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
     constexpr int UNR = 4;
     // `resume`: the range starts where the previous call's range ended (consecutive slot tiles of a row
     // with at most THREADS lists), so each list's lower end is remembered instead of searched again.
-    auto for_each_product = [&](auto what, auto dense_tag, uint32_t lo, uint32_t hi, bool whole, uint32_t c0, uint32_t s0,
+    // ones_tag: the partial products are ones (binary input, or the bit-setting pass): only row ids are read
+    auto for_each_product = [&](auto what, auto dense_tag, auto ones_tag, uint32_t lo, uint32_t hi, bool whole, uint32_t c0, uint32_t s0,
                                 bool resume) {
         constexpr int WHAT = decltype(what)::value;
+        constexpr bool ONES = decltype(ones_tag)::value || WHAT != CTA_ACCUM;
         for (uint32_t b0 = 0; b0 < deg; b0 += THREADS) {
             uint32_t sublen = 0, substart = 0;
             Acc a = Acc(0);
@@ -203,14 +212,14 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                             rel[u] = 0;
                             val[u] = Acc(0);
                             if (q[u] != 0xffffffffu) {
-                                if (WHAT == CTA_ACCUM && !binary) {
+                                if constexpr (!ONES) {
                                     // one load brings the row id and the value (the records the light rows gather)
                                     const ColRec<V> rec = static_cast<const ColRec<V>*>(P.at_rec)[q[u]];
                                     rel[u] = (uint32_t)rec.j - c0;
                                     val[u] = (Acc)rec.v;
                                 } else {
                                     rel[u] = (uint32_t)P.at_row[q[u]] - c0;
-                                    if (WHAT == CTA_ACCUM) val[u] = Acc(1);
+                                    val[u] = Acc(1);
                                 }
                             }
                         }
@@ -234,7 +243,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     Acc val[UNR];
 #pragma unroll
                     for (int u = 0; u < UNR; ++u) {
-                        if (WHAT == CTA_ACCUM && !binary) {
+                        if constexpr (!ONES) {
                             const ColRec<V> rec = recp[e + u * THREADS];
                             rel[u] = (uint32_t)rec.j - c0;
                             val[u] = (Acc)rec.v;
@@ -247,7 +256,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                     for (int u = 0; u < UNR; ++u) apply(what, dense_tag, rel[u], fa, val[u], s0);
                 }
                 for (; e < len; e += THREADS) {
-                    if (WHAT == CTA_ACCUM && !binary) {
+                    if constexpr (!ONES) {
                         const ColRec<V> rec = recp[e];
                         apply(what, dense_tag, (uint32_t)rec.j - c0, fa, (Acc)rec.v, s0);
                     } else {
@@ -273,7 +282,7 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
         if (!dense) {
             for (uint32_t w = tid; w < cwa; w += THREADS) bits[w] = 0;
             __syncthreads();
-            for_each_product(SET, NOT_DENSE, c0, c1, single_chunk, c0, 0u, false);
+            for_each_product(SET, NOT_DENSE, IS_DENSE, c0, c1, single_chunk, c0, 0u, false);
             uint32_t s = 0;
             for (uint32_t w = w0; w < w0 + per && w < cwa; ++w) s += __popc(bits[w]);
             uint32_t ex = block_exclusive_scan<uint32_t, THREADS>(s, scratch, &tot);
@@ -348,8 +357,14 @@ __global__ void __launch_bounds__(THREADS) rows_cta_kernel(PlanDev P, const int3
                 }
                 __syncthreads();
                 const bool resume = s0 > 0 && deg <= THREADS;
-                if (dense) for_each_product(ACC, IS_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
-                else for_each_product(ACC, NOT_DENSE, jlo, jhi, single_chunk && single_tile, c0, s0, resume);
+                const bool whole_row = single_chunk && single_tile;
+                if (binary) {  // (the tags are std::true_type / std::false_type: here "the products are ones")
+                    if (dense) for_each_product(ACC, IS_DENSE, IS_DENSE, jlo, jhi, whole_row, c0, s0, resume);
+                    else for_each_product(ACC, NOT_DENSE, IS_DENSE, jlo, jhi, whole_row, c0, s0, resume);
+                } else {
+                    if (dense) for_each_product(ACC, IS_DENSE, NOT_DENSE, jlo, jhi, whole_row, c0, s0, resume);
+                    else for_each_product(ACC, NOT_DENSE, NOT_DENSE, jlo, jhi, whole_row, c0, s0, resume);
+                }
                 for (uint32_t t = tid; t < s1 - s0; t += THREADS) {
                     if (!SPSYRK_IN_RANGE(ob + s0 + t < out_end, P.err)) continue;
                     const V cv = packed ? (V)((reinterpret_cast<const uint32_t*>(acc)[t >> 2] >> ((t & 3u) * 8u)) & 0xffu)
