@@ -169,8 +169,9 @@ spsyrk_status_t spsyrk_numeric_rows(spsyrk_plan_t plan, int64_t row_begin, int64
                                     void *cuda_stream);
 
 /*
- * One-pass mode: C_L without a separate symbolic pass, for callers that can afford a second, slightly larger
- * output buffer.  Every light row gets a slot sized by the number of its partial products (an upper bound of its
+ * One-pass mode: the product of spsyrk_symbolic + spsyrk_numeric (Section II-A, Algorithm 2 line 2: the lower
+ * triangle of A A^T, rows ascending in column) without a separate symbolic pass, for callers that can afford a
+ * second, slightly larger output buffer.  Every light row gets a slot sized by the number of its partial products (an upper bound of its
  * entries; the heavy rows, which find their structure in bitmaps anyway, get exact slots), the numeric kernel
  * that sorts a row's products computes the row into its slot and reports its count, and the rows are then moved
  * to their places.  The column lists are gathered once instead of twice.
